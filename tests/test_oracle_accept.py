@@ -1,0 +1,351 @@
+"""Pins of the oracle's acceptance walk against things other than itself: hand-computed cases,
+special cases with known outcomes, textbook linear speculative sampling, exact-rational
+resampling, brute-force greedy, and the closed form that the emitted tokens follow the target
+distribution (chi-square, with power checks)."""
+import json
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+from scipy import stats
+
+from oracle import ref
+from paper_2603_08899_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _logits_of(probs):
+    p = np.asarray(probs, dtype=np.float64)
+    with np.errstate(divide="ignore"):
+        lg = np.where(p > 0, np.log(np.where(p > 0, p, 1.0)), -1e4)
+    return torch.from_numpy(lg)
+
+
+@pytest.mark.parametrize("case", json.load(open(os.path.join(GOLDEN, "accept_hand_cases.json")))["cases"],
+                         ids=lambda c: c["name"])
+def test_hand_computed_cases(case):
+    tl = _logits_of(case["p"])[None]
+    dl = _logits_of(case["q"])[None]
+    o = ref.tree_accept(tl, dl, torch.tensor([case["tokens"]]), torch.tensor([case["parent"]]),
+                        torch.tensor([case["owner"]]), torch.tensor([case["u"]], dtype=torch.float64),
+                        temperature=1.0, sibling_mode=case["mode"])
+    assert o["status"].tolist() == [0]
+    assert o["accept_len"].tolist() == [case["accept_len"]]
+    n = len(case["path"])
+    assert o["path"][0, :n].tolist() == case["path"] and (o["path"][0, n:] == -1).all()
+    assert o["next_token"].tolist() == [case["next_token"]]
+    assert o["future_row"].tolist() == [case["future_row"]]
+    assert o["counters"][0, :2].tolist() == [case["tests"], case["rejections"]]
+
+
+def _random_case(T=12, V=50, B=4, seed=3, draft="independent", tree="random", C=3, dtype=torch.float32):
+    cfg = inputs.VerifyConfig("a", B=B, L=1, Hq=2, Hkv=1, D=16, T=T, C=C, S=0, V=V, prefix=4, tree=tree,
+                              kv_dtype=torch.float32, logit_dtype=dtype, sigma_logit=2.0, draft=draft,
+                              temperatures=(1.0,), seed=seed, max_depth=4, fanout=(1, 3))
+    parent, owner = inputs.trees(cfg)
+    tl, dl = inputs.logits(cfg)
+    tok = inputs.draft_tokens(cfg, parent, dl, 1.0)
+    u = inputs.uniforms(cfg)
+    return cfg, parent, owner, tl, dl, tok, u
+
+
+def test_identical_distributions_always_accept_first_child():
+    cfg, parent, owner, tl, dl, tok, u = _random_case(seed=4)
+    o = ref.tree_accept(tl, tl.clone(), tok, parent, owner, u, temperature=0.8)
+    for b in range(cfg.B):
+        par = parent[b].tolist()
+        cur, path = 0, [0]
+        while True:
+            kids = [i for i in range(cfg.T) if par[i] == cur]
+            if not kids:
+                break
+            cur = kids[0]
+            path.append(cur)
+        assert o["accept_len"][b].item() == len(path) - 1
+        assert o["path"][b, :len(path)].tolist() == path
+        p = torch.softmax(tl[b, cur].double() / 0.8, 0).numpy()
+        cdf = np.cumsum(p)
+        want = int(np.searchsorted(cdf, float(u[b, 0]) * cdf[-1], side="right"))
+        assert o["next_token"][b].item() == want
+        assert o["counters"][b, 1].item() == 0
+
+
+def _linear_speculative_sampling(p_rows, q_rows, toks, u):
+    """Textbook linear speculative sampling (accept draft i while u_i < p_i(x_i)/q_i(x_i); at the first
+    rejection sample from norm(max(p_i - q_i, 0)); if all accepted sample from the next target row)."""
+    K = len(toks)
+    for i in range(K):
+        x = toks[i]
+        if u[i + 1] < p_rows[i][x] / q_rows[i][x]:
+            continue
+        res = np.maximum(p_rows[i] - q_rows[i], 0.0)
+        cdf = np.cumsum(res)
+        return i, int(np.searchsorted(cdf, u[0] * cdf[-1], side="right"))
+    cdf = np.cumsum(p_rows[K])
+    return K, int(np.searchsorted(cdf, u[0] * cdf[-1], side="right"))
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_chain_tree_is_linear_speculative_sampling(mode):
+    cfg, parent, owner, tl, dl, tok, u = _random_case(T=9, V=40, B=16, seed=5, draft="noise", tree="chain", C=0)
+    o = ref.tree_accept(tl, dl, tok, parent, owner, u, temperature=1.0, sibling_mode=mode)
+    lens = []
+    for b in range(cfg.B):
+        p = torch.softmax(tl[b].double(), -1).numpy()
+        q = torch.softmax(dl[b].double(), -1).numpy()
+        n_acc, nxt = _linear_speculative_sampling(p, q, tok[b, 1:].tolist(), u[b].double().numpy())
+        assert o["accept_len"][b].item() == n_acc
+        assert o["next_token"][b].item() == nxt
+        lens.append(n_acc)
+    assert 0 < sum(lens) < 8 * cfg.B          # the case exercises both outcomes
+
+
+def test_resample_against_exact_rationals():
+    """Residual and inverse CDF in exact rational arithmetic on a 12-token vocabulary."""
+    rng = np.random.default_rng(7)
+    V = 12
+    for trial in range(40):
+        pi = rng.integers(0, 9, V)
+        qi = rng.integers(1, 9, V)
+        pi[rng.integers(V)] += 1
+        p = [Fraction(int(a), int(pi.sum())) for a in pi]
+        q = [Fraction(int(a), int(qi.sum())) for a in qi]
+        x = int(rng.integers(V))                       # the (rejected) child token
+        u0 = Fraction(int(rng.integers(0, 1 << 20)), 1 << 20)
+        ratio = p[x] / q[x]
+        u1 = float(min(Fraction(999, 1000), ratio + Fraction(1, 64)))   # just above the ratio -> reject
+        if ratio >= Fraction(63, 64):
+            continue
+        res = [max(a - b, Fraction(0)) for a, b in zip(p, q)]
+        tot = sum(res)
+        c, want = Fraction(0), None
+        for k in range(V):
+            c += res[k]
+            if c > u0 * tot:
+                want = k
+                break
+        # keep away from cell edges, where double rounding may legitimately differ
+        edges = np.cumsum([float(r / tot) for r in res])
+        if np.min(np.abs(edges - float(u0))) < 1e-9:
+            continue
+        tl = _logits_of([[float(a) for a in p]] * 2)[None]
+        dl = _logits_of([[float(a) for a in q]] * 2)[None]
+        o = ref.tree_accept(tl, dl, torch.tensor([[0, x]]), torch.tensor([[-1, 0]]), None,
+                            torch.tensor([[float(u0), u1]], dtype=torch.float64))
+        assert o["accept_len"].tolist() == [0]
+        assert o["next_token"].tolist() == [want], (trial, want)
+
+
+def test_greedy_equals_bruteforce_longest_matching_path():
+    for seed in range(6):
+        cfg, parent, owner, tl, dl, tok, u = _random_case(T=14, V=6, B=8, seed=20 + seed, dtype=torch.bfloat16)
+        # small vocabulary + bf16 => plenty of matches and of ties
+        tok = torch.randint(0, cfg.V, tok.shape, generator=torch.Generator().manual_seed(seed), dtype=torch.int32)
+        o = ref.tree_accept(tl, None, tok, parent, owner, None, temperature=0.0)
+        for b in range(cfg.B):
+            par = parent[b].tolist()
+            am = [int(np.argmax(tl[b, i].double().numpy())) for i in range(cfg.T)]   # numpy: first maximum
+            best, best_path = 0, [0]
+            for leaf in range(cfg.T):
+                chain = []
+                a = leaf
+                while a >= 0:
+                    chain.append(a)
+                    a = par[a]
+                chain.reverse()
+                ok = [0]
+                for node in chain[1:]:
+                    if tok[b, node].item() == am[par[node]]:
+                        ok.append(node)
+                    else:
+                        break
+                if len(ok) - 1 > best or (len(ok) - 1 == best and ok[-1] < best_path[-1]):
+                    best, best_path = len(ok) - 1, ok
+            assert o["accept_len"][b].item() == best
+            assert o["path"][b, :best + 1].tolist() == best_path
+            assert o["next_token"][b].item() == am[best_path[-1]]
+
+
+def test_future_row_falls_back_to_nearest_ancestor():
+    # chain of 5, contemplate rows on nodes 0 and 2 only; identical logits => walk reaches node 4
+    T, V = 5, 8
+    tl = torch.randn(1, T, V, dtype=torch.float64)
+    tok = torch.randint(0, V, (1, T), dtype=torch.int32)
+    parent = torch.from_numpy(inputs.chain_tree(T))[None]
+    o = ref.tree_accept(tl, tl.clone(), tok, parent, torch.tensor([[0, 2]]), torch.full((1, T), 0.5, dtype=torch.float64))
+    assert o["accept_len"].tolist() == [4] and o["future_row"].tolist() == [T + 1]
+    o = ref.tree_accept(tl, tl.clone(), tok, parent, torch.tensor([[3, 1]]), torch.full((1, T), 0.5, dtype=torch.float64))
+    assert o["future_row"].tolist() == [T + 0]
+    o = ref.tree_accept(tl, tl.clone(), tok, parent, torch.zeros(1, 0, dtype=torch.int32), torch.full((1, T), 0.5, dtype=torch.float64))
+    assert o["future_row"].tolist() == [-1]
+
+
+def test_input_errors_are_reported():
+    cfg, parent, owner, tl, dl, tok, u = _random_case(seed=9, B=3)
+    bad_tok = tok.clone()
+    bad_tok[1, 2] = cfg.V
+    assert ref.tree_accept(tl, dl, bad_tok, parent, owner, u)["status"].tolist() == [0, ref.ST_BAD_TOKEN, 0]
+    dup = tok.clone()
+    par = parent[2].tolist()
+    sib = [(i, j) for i in range(1, cfg.T) for j in range(i + 1, cfg.T) if par[i] == par[j]]
+    i, j = sib[0]
+    dup[2, j] = dup[2, i]
+    o = ref.tree_accept(tl, dl, dup, parent, owner, u, sibling_mode=1)
+    assert o["status"].tolist() == [0, 0, ref.ST_DUP_SIBLING] and o["next_token"][2].item() == -1
+    assert ref.tree_accept(tl, dl, dup, parent, owner, u, sibling_mode=0)["status"].tolist() == [0, 0, 0]
+    nan = tl.clone()
+    nan[0, 3, 5] = float("nan")
+    assert ref.tree_accept(nan, dl, tok, parent, owner, u)["status"].tolist() == [ref.ST_NONFINITE, 0, 0]
+
+
+# ------------------------------------------------------------------ distribution test
+V16 = 16
+PARENT10 = np.array([-1, 0, 0, 0, 1, 1, 2, 2, 3, 3], dtype=np.int32)    # root -> 3 children -> 2 children each
+
+
+def _tables(seed):
+    rng = np.random.default_rng(seed)
+
+    def soft(x):
+        e = np.exp(x - x.max(-1, keepdims=True))
+        return e / e.sum(-1, keepdims=True)
+    P0, Q0 = soft(rng.normal(0, 1.5, V16)), soft(rng.normal(0, 1.5, V16))
+    P1, Q1 = soft(rng.normal(0, 1.5, (V16, V16))), soft(rng.normal(0, 1.5, (V16, V16)))
+    P2 = soft(rng.normal(0, 1.5, (V16, V16, V16)))
+    return P0, Q0, P1, Q1, P2
+
+
+def _draw(rng, q, n, mode):
+    if mode == 0:
+        return rng.choice(V16, size=n, p=q)
+    out, qq = [], q.copy()
+    for _ in range(n):
+        x = rng.choice(V16, p=qq / qq.sum())
+        out.append(x)
+        qq[x] = 0.0
+    return np.array(out)
+
+
+def _trials(N, draw_mode, seed):
+    """N independent verification steps on the 10-node tree with context-dependent rows."""
+    P0, Q0, P1, Q1, P2 = _tables(1234)
+    rng = np.random.default_rng(seed)
+    tok = np.zeros((N, 10), dtype=np.int32)
+    tl = np.zeros((N, 10, V16))
+    dl = np.zeros((N, 10, V16))
+    for n in range(N):
+        t1 = _draw(rng, Q0, 3, draw_mode)
+        tok[n, 1:4] = t1
+        tl[n, 0], dl[n, 0] = P0, Q0
+        for i, a in enumerate(t1):
+            node = 1 + i
+            tl[n, node], dl[n, node] = P1[a], Q1[a]
+            t2 = _draw(rng, Q1[a], 2, draw_mode)
+            for j, c in enumerate(t2):
+                leaf = 4 + 2 * i + j
+                tok[n, leaf] = c
+                tl[n, leaf] = P2[a, c]
+                dl[n, leaf] = P2[a, c]
+    u = rng.random((N, 10))
+    return (torch.from_numpy(np.log(tl)), torch.from_numpy(np.log(dl)), torch.from_numpy(tok),
+            torch.from_numpy(np.tile(PARENT10, (N, 1))), torch.from_numpy(u), (P0, P1))
+
+
+def _chi2_pvalues(first, second_given, P0, P1):
+    """first: emitted first tokens; second_given: list of (t1, t2) for steps that accepted >= 1 node."""
+    N = len(first)
+    obs = np.bincount(first, minlength=V16)
+    p_first = stats.chisquare(obs, N * P0).pvalue
+    chi, dof = 0.0, 0
+    pairs = np.asarray(second_given)
+    for a in range(V16):
+        sel = pairs[pairs[:, 0] == a, 1]
+        if len(sel) < 200:
+            continue
+        exp = len(sel) * P1[a]
+        o = np.bincount(sel, minlength=V16).astype(float)
+        small = exp < 5                                       # pool sparse cells
+        if small.sum() > 0:
+            o = np.append(o[~small], o[small].sum())
+            exp = np.append(exp[~small], exp[small].sum())
+        chi += ((o - exp) ** 2 / exp).sum()
+        dof += len(exp) - 1
+    return p_first, stats.chi2.sf(chi, dof)
+
+
+def _emitted(o, tok):
+    a = o["accept_len"].numpy()
+    path = o["path"].numpy()
+    nxt = o["next_token"].numpy()
+    tok = tok.numpy()
+    N = len(a)
+    first = np.where(a >= 1, tok[np.arange(N), np.maximum(path[:, 1], 0)], nxt)
+    second = []
+    for n in np.nonzero(a >= 1)[0]:
+        t2 = tok[n, path[n, 2]] if a[n] >= 2 else nxt[n]
+        second.append((first[n], t2))
+    return first, second
+
+
+N_TRIALS = 60000
+
+
+@pytest.mark.parametrize("mode", [1, 0])
+def test_emitted_tokens_follow_the_target_distribution(mode):
+    """Speculative sampling preserves the target model's sampling distribution: the first emitted
+    token is distributed as the root's target row, the second (given the first was an accepted
+    draft) as the target row of that node."""
+    tl, dl, tok, parent, u, (P0, P1) = _trials(N_TRIALS, mode, seed=99 + mode)
+    o = ref.tree_accept(tl, dl, tok, parent, None, u, temperature=1.0, sibling_mode=mode)
+    assert (o["status"] == 0).all()
+    first, second = _emitted(o, tok)
+    p_first, p_second = _chi2_pvalues(first, second, P0, P1)
+    assert p_first > 1e-4 and p_second > 1e-4, (p_first, p_second)
+    assert 0.3 < (o["accept_len"] >= 1).float().mean() < 0.99
+
+
+def test_distribution_test_has_power_against_the_wrong_sibling_rule():
+    """Children drawn without replacement but verified with the i.i.d. rule (q not updated after a
+    rejection) must be caught by the same chi-square test."""
+    tl, dl, tok, parent, u, (P0, P1) = _trials(N_TRIALS, 1, seed=100)
+    o = ref.tree_accept(tl, dl, tok, parent, None, u, temperature=1.0, sibling_mode=0)
+    first, second = _emitted(o, tok)
+    p_first, _ = _chi2_pvalues(first, second, P0, P1)
+    assert p_first < 1e-6, p_first
+
+
+def _python_walk(tl, dl, tok, parent, u, drop_residual=False):
+    """A separate, deliberately breakable restatement of the root-level step (first emitted token only)."""
+    p = np.exp(tl[0])
+    q = np.exp(dl[0])
+    p, q = p / p.sum(), q / q.sum()
+    for c in np.nonzero(parent == 0)[0]:
+        x = tok[c]
+        if u[c] < p[x] / q[x]:
+            return x
+        if not drop_residual:
+            p = np.maximum(p - q, 0)
+            p = p / p.sum()
+        q = q.copy()
+        q[x] = 0
+        q = q / q.sum()
+    cdf = np.cumsum(p)
+    return int(np.searchsorted(cdf, u[0] * cdf[-1], side="right"))
+
+
+def test_distribution_test_has_power_against_a_dropped_residual_step():
+    N = 20000
+    tl, dl, tok, parent, u, (P0, P1) = _trials(N, 1, seed=101)
+    tln, dln, tokn, un = tl.numpy(), dl.numpy(), tok.numpy(), u.numpy()
+    good = np.array([_python_walk(tln[n], dln[n], tokn[n], PARENT10, un[n]) for n in range(N)])
+    broken = np.array([_python_walk(tln[n], dln[n], tokn[n], PARENT10, un[n], drop_residual=True) for n in range(N)])
+    assert stats.chisquare(np.bincount(good, minlength=V16), N * P0).pvalue > 1e-4
+    assert stats.chisquare(np.bincount(broken, minlength=V16), N * P0).pvalue < 1e-6
+    # and the separate restatement agrees with the oracle on the first emitted token
+    o = ref.tree_accept(tl, dl, tok, parent, None, u, temperature=1.0, sibling_mode=1)
+    first, _ = _emitted(o, tok)
+    assert (first == good).all()
