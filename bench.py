@@ -1,0 +1,422 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verification step (L x tree attention + acceptance + KV compaction).
+
+    python bench.py --gpus 1 --steps 20 --warmup 3                # this library, on the GPU
+    python bench.py --impl reference --steps 2 --warmup 1         # the fp64 CPU oracle on the host cores
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
+
+Prints ONE JSON line.  Workload: seeded synthetic inputs shaped like a batched Llama-3.1-8B
+verification step (32 sequences, ragged prefixes, 60-node trees + 4 contemplate rows).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2603_08899_b200 import inputs  # noqa: E402
+
+METRIC = "verify_steps_per_sec"
+UNIT = "steps/s"
+
+
+# ----------------------------------------------------------------------------- byte / flop model
+def attention_bytes_per_layer(cfg, plen):
+    """Algorithmic HBM bytes of one attention launch: every K and V row of every sequence read once
+    (prefix + the R rows' own slots), the soft-prompt K/V once, Q read and O written once."""
+    es = 2 if cfg.kv_dtype == torch.bfloat16 else 4
+    row = cfg.Hkv * cfg.D * es
+    kv = 2 * row * int((plen.to(torch.int64) + cfg.R).sum())
+    soft = 2 * row * cfg.S
+    qo = 2 * cfg.B * cfg.R * cfg.Hq * cfg.D * es
+    return kv + soft + qo
+
+
+def attention_flops_per_layer(cfg, plen):
+    keys = int((plen.to(torch.int64) + cfg.R + cfg.S).sum())
+    return 4 * cfg.R * cfg.Hq * cfg.D * keys
+
+
+def step_bytes(cfg, plen, accept_len_mean):
+    es = 2 if cfg.logit_dtype == torch.bfloat16 else 4
+    logits = 2 * cfg.B * cfg.T * cfg.V * es
+    row = cfg.Hkv * cfg.D * (2 if cfg.kv_dtype == torch.bfloat16 else 4)
+    compact = int(2 * 2 * accept_len_mean * row * cfg.L * cfg.B)
+    return cfg.L * attention_bytes_per_layer(cfg, plen) + logits + compact
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
+
+
+def profile_traffic(kernel):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if there is one."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(p):
+        return json.load(open(p)).get(kernel)
+    return None
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- CPU oracle leg
+def oracle_prepare(cfg, target_visits=100e6):
+    """Inputs of the bounded oracle sample (generation is not timed).  The number of sampled attention
+    rows is set so that the sample visits about `target_visits` (row, key) pairs: ~10 s on 8 cores."""
+    parent, owner = inputs.trees(cfg)
+    plen = inputs.prefix_lens(cfg)
+    nseq = min(cfg.B, 4)
+    sub = inputs.scaled(cfg, B=nseq)
+    sp = {"cfg": cfg, "nseq": nseq, "plen_all": plen, "parent": parent[:nseq].contiguous(),
+          "owner": owner[:nseq].contiguous(), "plen": plen[:nseq].contiguous()}
+    sp["seq_start"], n_slots = inputs.cache_layout(sub, sp["plen"])
+    sp["t"] = inputs.layer_tensors(sub, 0, n_slots)
+    rows_per_seq = max(8, min(cfg.R * cfg.Hq, int(target_visits / max(1, int(sp["plen"].sum()) + nseq * cfg.R))))
+    g = torch.Generator().manual_seed(11)
+    sp["sel"] = [(b, int(torch.randint(0, cfg.R, (1,), generator=g)), int(torch.randint(0, cfg.Hq, (1,), generator=g)))
+                 for b in range(nseq) for _ in range(rows_per_seq)]
+    sp["tl"], sp["dl"] = inputs.logits(sub)
+    sp["tok"] = inputs.draft_tokens(sub, sp["parent"], sp["dl"], 1.0)
+    sp["u"] = inputs.uniforms(sub)
+    return sp
+
+
+def oracle_sample(sp):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload and scales the result
+    to one whole step.  Sample: a few hundred (row, head) outputs of layer 0 for up to 4 sequences
+    (attention cost is proportional to the visible keys, which the scaling uses), the acceptance walk
+    of those sequences at full vocabulary, and the compaction of one layer."""
+    from oracle import ref
+    cfg, nseq, t = sp["cfg"], sp["nseq"], sp["t"]
+    t0 = time.perf_counter()
+    ref.tree_attention_rows(t["q"], t["k_cache"], t["v_cache"], sp["seq_start"], sp["plen"], t["k_soft"], t["v_soft"],
+                            sp["parent"], sp["owner"], sp["sel"])
+    t_attn = time.perf_counter() - t0
+    keys_sampled = sum(int(sp["plen"][b]) + cfg.R + (cfg.S if r >= cfg.T else 0) for b, r, _ in sp["sel"])
+    keys_step = cfg.L * cfg.Hq * sum((int(p) + cfg.R) * cfg.R + cfg.S * cfg.C for p in sp["plen_all"])
+    t0 = time.perf_counter()
+    o = ref.tree_accept(sp["tl"], sp["dl"], sp["tok"], sp["parent"], sp["owner"], sp["u"], temperature=1.0)
+    t_acc = time.perf_counter() - t0
+    kc, vc = t["k_cache"].clone(), t["v_cache"].clone()
+    t0 = time.perf_counter()
+    ref.kv_compact([kc], [vc], sp["seq_start"], sp["plen"], o["accept_len"], o["path"])
+    t_cmp = time.perf_counter() - t0
+    est = t_attn * keys_step / keys_sampled + (t_acc + t_cmp * cfg.L) * cfg.B / nseq
+    return {"step_seconds_estimate": est, "sample_seconds": t_attn + t_acc + t_cmp, "cores": ref.num_threads(),
+            "sample": f"{len(sp['sel'])} attention output rows of layer 0 over {nseq} sequences ({keys_sampled} key "
+                      f"visits of {keys_step} per step), acceptance of {nseq} sequences at full vocabulary, "
+                      f"compaction of 1 layer; scaled linearly to {cfg.L} layers x {cfg.B} sequences"}
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sp = oracle_prepare(cfg, target_visits=25e6)
+    for i in range(args.warmup):
+        oracle_sample(sp)
+    t0 = time.perf_counter()
+    res = [oracle_sample(sp) for i in range(args.steps)]
+    wall = time.perf_counter() - t0
+    est = statistics.mean(r["step_seconds_estimate"] for r in res)
+    value = 1.0 / est
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "note": "oracle timed on a bounded sample, scaled to a whole step",
+                       "sample_wall_seconds": wall},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": res[0]["cores"], "kind": "oracle",
+                             "sample": res[0]["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- GPU leg
+def build_workload(cfg, device, rank):
+    from paper_2603_08899_b200.step import VerifyStep
+    if rank:
+        cfg = inputs.scaled(cfg, seed=cfg.seed + 1000 * rank)      # every rank its own batch (weak scaling)
+    parent, owner = inputs.trees(cfg)
+    plen = inputs.prefix_lens(cfg)
+    seq_start, n_slots = inputs.cache_layout(cfg, plen)
+    q, k, v, ks, vs, out = [], [], [], [], [], []
+    for l in range(cfg.L):
+        t = inputs.layer_tensors(cfg, l, n_slots, device=device)
+        q.append(t["q"]); k.append(t["k_cache"]); v.append(t["v_cache"]); ks.append(t["k_soft"]); vs.append(t["v_soft"])
+        out.append(torch.empty_like(t["q"]))
+    tl, dl = inputs.logits(cfg, device=device)
+    tok = inputs.draft_tokens(cfg, parent, dl, 1.0)
+    u = inputs.uniforms(cfg)
+    step = VerifyStep(cfg, n_slots, device=device)
+    step.bind(q, k, v, ks if cfg.S else None, vs if cfg.S else None, out, seq_start.to(device), plen.to(device),
+              parent.to(device), owner.to(device) if cfg.C else None, tl, dl, tok.to(device), u.to(device))
+    host = {"parent": parent, "owner": owner, "plen": plen, "seq_start": seq_start, "tok": tok, "u": u}
+    return cfg, step, host
+
+
+def spot_check(cfg, step, host):
+    """Before timing: the acceptance outputs of the first sequences against the oracle (cheap)."""
+    from oracle import ref
+    n = min(cfg.B, 2)
+    o = ref.tree_accept(step.tl[:n].cpu(), step.dl[:n].cpu(), host["tok"][:n], host["parent"][:n], host["owner"][:n],
+                        host["u"][:n], temperature=1.0)
+    ok = True
+    for b in range(n):
+        same = step.accept_len[b].item() == o["accept_len"][b].item() and \
+            step.next_token[b].item() == o["next_token"][b].item()
+        ok &= bool(same or o["ratio_margin"][b].item() < 1e-5 or o["resample_margin"][b].item() < 1e-5)
+    return ok
+
+
+def run_ours(args, cfg):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; this library has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    from paper_2603_08899_b200 import binding as cb
+    from paper_2603_08899_b200 import step as step_mod
+
+    cfg, step, host = build_workload(cfg, device, rank)
+    plen = host["plen"]
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----
+    for _ in range(args.warmup):
+        step.status.zero_()
+        step.run(1.0)
+    torch.cuda.synchronize()
+    checked = spot_check(cfg, step, host) if rank == 0 else True
+    status_ok = bool((step.status == 0).all().item())
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(args.steps):
+        ev[i][0].record()
+        cb.confu_tree_plan(step.ctx, step.dims, step.seq_start, step.prefix_len, step.parent, step.con_owner,
+                           step.plan, step.status)
+        ev[i][1].record()
+        for l in range(cfg.L):
+            cb.confu_tree_attention(step.ctx, step.dims, step.q[l], step.k[l], step.v[l], step.n_slots,
+                                    step.seq_start, step.prefix_len, step.ks[l] if step.ks else None,
+                                    step.vs[l] if step.vs else None, None, None, step.plan, step.out[l], None,
+                                    step.status)
+        ev[i][2].record()
+        step.run_accept(1.0)
+        ev[i][3].record()
+        step.run_compact()
+        ev[i][4].record()
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = t_begin.elapsed_time(t_end)
+    if dist is not None:
+        tt = torch.tensor([total_ms], device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = tt.item()
+    ms_step = total_ms / args.steps
+    part = lambda a, b: statistics.mean(ev[i][a].elapsed_time(ev[i][b]) for i in range(args.steps))  # noqa: E731
+    ms_plan, ms_attn, ms_acc, ms_cmp = part(0, 1), part(1, 2), part(2, 3), part(3, 4)
+    alen = step.accept_len.float().mean().item()
+
+    # ---- end to end: this step's inputs come from pinned host memory, results go back ----
+    h = {"q": [t.cpu().pin_memory() for t in step.q],
+         "krows": [], "vrows": [],
+         "tl": step.tl.cpu().pin_memory(), "dl": step.dl.cpu().pin_memory(),
+         "tok": host["tok"].pin_memory(), "u": host["u"].pin_memory(), "parent": host["parent"].pin_memory(),
+         "owner": host["owner"].pin_memory()}
+    R = cfg.R
+    idx = torch.cat([torch.arange(int(host["seq_start"][b]) + int(plen[b]), int(host["seq_start"][b]) + int(plen[b]) + R)
+                     for b in range(cfg.B)]).to(device)
+    for l in range(cfg.L):
+        h["krows"].append(step.k[l][idx].view(cfg.B, R, cfg.Hkv, cfg.D).cpu().pin_memory())
+        h["vrows"].append(step.v[l][idx].view(cfg.B, R, cfg.Hkv, cfg.D).cpu().pin_memory())
+    d_krows = torch.empty_like(h["krows"][0], device=device)
+    d_vrows = torch.empty_like(h["vrows"][0], device=device)
+    res_host = {k: torch.empty_like(getattr(step, k), device="cpu").pin_memory()
+                for k in ("accept_len", "path", "next_token", "future_row", "new_prefix_len", "status")}
+    h2d = sum(t.numel() * t.element_size() for t in h["q"] + h["krows"] + h["vrows"]) + \
+        sum(h[k].numel() * h[k].element_size() for k in ("tl", "dl", "tok", "u", "parent", "owner"))
+    d2h = sum(t.numel() * t.element_size() for t in res_host.values())
+
+    def e2e_step():
+        step.parent.copy_(h["parent"], non_blocking=True)
+        if cfg.C:
+            step.con_owner.copy_(h["owner"], non_blocking=True)
+        step.tokens.copy_(h["tok"], non_blocking=True)
+        step.uniforms.copy_(h["u"], non_blocking=True)
+        cb.confu_tree_plan(step.ctx, step.dims, step.seq_start, step.prefix_len, step.parent, step.con_owner,
+                           step.plan, step.status)
+        for l in range(cfg.L):
+            step.q[l].copy_(h["q"][l], non_blocking=True)
+            d_krows.copy_(h["krows"][l], non_blocking=True)
+            d_vrows.copy_(h["vrows"][l], non_blocking=True)
+            cb.confu_kv_append(step.ctx, step.dims, d_krows, d_vrows, step.k[l], step.v[l], step.seq_start,
+                               step.prefix_len)
+            cb.confu_tree_attention(step.ctx, step.dims, step.q[l], step.k[l], step.v[l], step.n_slots,
+                                    step.seq_start, step.prefix_len, step.ks[l] if step.ks else None,
+                                    step.vs[l] if step.vs else None, None, None, step.plan, step.out[l], None,
+                                    step.status)
+        step.tl.copy_(h["tl"], non_blocking=True)
+        step.dl.copy_(h["dl"], non_blocking=True)
+        step.run_accept(1.0)
+        step.run_compact()
+        for k, t in res_host.items():
+            t.copy_(getattr(step, k), non_blocking=True)
+
+    n_e2e = max(2, min(args.steps, 5))
+    e2e_step()
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n_e2e):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tt = torch.tensor([e2e_ms], device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = tt.item()
+    e2e_value = world * n_e2e / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    a_bytes = attention_bytes_per_layer(cfg, plen)
+    a_flops = attention_flops_per_layer(cfg, plen)
+    attn_launch_s = ms_attn * 1e-3 / cfg.L
+    achieved = a_bytes / attn_launch_s / 1e9
+    sbytes = step_bytes(cfg, plen, alen)
+    kname = "attention_tc" if step_mod.ATTENTION_KERNELS_PER_LAYER > 1 else "attention_generic"
+    cpu = oracle_sample(oracle_prepare(cfg)) if not args.no_cpu_baseline else None
+    line = {
+        "metric": METRIC, "value": world * args.steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "layers": cfg.L, "heads": f"{cfg.Hq}q/{cfg.Hkv}kv", "head_dim": cfg.D,
+                   "tree_rows": cfg.T, "contemplate_rows": cfg.C, "soft_prompt": cfg.S, "vocab": cfg.V,
+                   "prefix": "ragged U[512,16384]" if isinstance(cfg.prefix, tuple) else cfg.prefix,
+                   "sum_prefix": int(plen.sum()), "temperature": 1.0,
+                   "l2": "inputs larger than L2 (every layer has its own KV; no flush needed)",
+                   "parallelism": f"replicas x{world}, sequences sharded, no collective",
+                   "parts_ms": {"plan": ms_plan, "attention": ms_attn, "accept": ms_acc, "compact": ms_cmp},
+                   "step_bytes": sbytes, "step_gbs": sbytes / (ms_step * 1e-3) / 1e9,
+                   "step_frac_of_hbm_roofline": sbytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                   "mean_accept_len": alen, "status_ok": status_ok, "spot_check_vs_oracle": checked},
+        "roofline": {"bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": profile_traffic(kname),
+                     "peak_source": peaks["source"], "bytes_per_launch": a_bytes, "launch_ms": attn_launch_s * 1e3,
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "tensor_tflops": a_flops / attn_launch_s / 1e12,
+                     "tensor_frac_of_bf16_peak": a_flops / attn_launch_s / 1e12 / peaks["bf16_tflops"]},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / n_e2e, "steps": n_e2e,
+                "note": "per step: Q, the R rows' K/V (all layers), both logit matrices, tree arrays and uniforms "
+                        "copied from pinned host memory; results copied back; the prefix KV cache is resident state"},
+        "gpu_launches": args.steps * step.launches_per_step(),
+        "clocks": clocks,
+    }
+    if cpu is not None:
+        line["cpu_baseline"] = {"value": 1.0 / cpu["step_seconds_estimate"], "unit": UNIT, "cores": cpu["cores"],
+                                "kind": "oracle", "sample": cpu["sample"], "sample_seconds": cpu["sample_seconds"]}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="batch32", choices=list(inputs.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = inputs.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

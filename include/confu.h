@@ -1,0 +1,212 @@
+/*
+ * confu.h -- C ABI of the B200 (sm_100a) tree-verification library.
+ *
+ * The library implements the target model's verification step of ConFu-style
+ * speculative decoding (ConFu, Sec. 2 "Preliminaries" steps 2-4 and the paragraph
+ * on token trees; Sec. 3.1 "Capture Future with Contemplate Tokens", Fig. 3):
+ *
+ *   confu_tree_attention   tree-masked attention of the draft-tree rows and the
+ *                          contemplate rows over prefix KV, soft-prompt KV and the
+ *                          tree's own KV (one layer per call)
+ *   confu_tree_accept      tree speculative-sampling acceptance over full-vocabulary
+ *                          logits, residual resampling, accepted path, future row
+ *   confu_kv_compact       keeps the accepted path's KV (all layers, one call)
+ *
+ * Conventions
+ *   - every function returns an int: 0 = CONFU_OK, negative = an error detected on
+ *     the host before anything was enqueued (see confu_status_string);
+ *   - "device" pointers are CUDA device pointers of the context's device, "host"
+ *     pointers are ordinary host memory; every device pointer must be 16-byte
+ *     aligned; the caller owns every buffer it passes, for the whole time the
+ *     enqueued work runs;
+ *   - work is enqueued on the given stream (a cudaStream_t passed as void*); no call
+ *     synchronises the host with the device and none allocates device memory except
+ *     confu_create / confu_destroy;
+ *   - data-dependent problems (a malformed tree, an out-of-range token, a
+ *     non-finite logit, a bounded device-side wait that ran out) never trap: the
+ *     kernels write a positive code into status[b] (int32, device, one per sequence).
+ *     The library only ever writes non-zero codes there, so clear it before a step.
+ *     A sequence with a non-zero status has unspecified outputs.
+ *
+ * Row and slot conventions
+ *   T tree rows (row 0 = root = the token emitted by the previous step), then C
+ *   contemplate rows; R = T + C <= 64.  parent[b][0] = -1 and 0 <= parent[b][i] < i.
+ *   con_owner[b][k] in [0,T) is the tree node that contemplate row T+k sits behind.
+ *   A layer's cache pool is [n_slots][Hkv][D]; sequence b owns slots
+ *   seq_start[b] .. seq_start[b] + prefix_len[b] + R - 1: its prefix, then the K/V of
+ *   its R query rows (written there by the caller before confu_tree_attention).
+ */
+#ifndef CONFU_H
+#define CONFU_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct confu_ctx confu_ctx;
+
+/* return codes (host side) */
+enum {
+    CONFU_OK = 0,
+    CONFU_ERR_ARG = -1,          /* null pointer / negative size / bad enum */
+    CONFU_ERR_SHAPE = -2,        /* Hq % Hkv != 0, D not in {64,128}, T < 1, ... */
+    CONFU_ERR_ALIGN = -3,        /* a device pointer is not 16-byte aligned */
+    CONFU_ERR_WORKSPACE = -4,    /* workspace missing or too small */
+    CONFU_ERR_UNSUPPORTED = -5,  /* e.g. R > 64 */
+    CONFU_ERR_CUDA = -6          /* a CUDA call failed: see confu_last_cuda_error */
+};
+
+/* per-sequence status codes written by the kernels (device side) */
+enum {
+    CONFU_ST_OK = 0,
+    CONFU_ST_BAD_PARENT = 1,
+    CONFU_ST_BAD_OWNER = 2,
+    CONFU_ST_BAD_TOKEN = 3,
+    CONFU_ST_DUP_SIBLING = 4,
+    CONFU_ST_NONFINITE = 5,
+    CONFU_ST_TIMEOUT = 6,        /* a bounded wait inside a kernel gave up */
+    CONFU_ST_DEGENERATE = 7,     /* residual distribution had no mass; target row used instead */
+    CONFU_ST_TOO_DEEP = 8        /* accepted path longer than CONFU_MAX_DEPTH */
+};
+
+enum { CONFU_BF16 = 0, CONFU_F32 = 1 };
+
+#define CONFU_MAX_ROWS  64      /* R = T + C */
+#define CONFU_MAX_DEPTH 63      /* path buffers hold CONFU_MAX_DEPTH + 1 node ids */
+
+typedef struct {
+    int32_t B;          /* sequences */
+    int32_t Hq, Hkv;    /* query / KV heads, Hq % Hkv == 0 */
+    int32_t D;          /* head dim: 64 or 128 */
+    int32_t T, C;       /* tree rows (root included), contemplate rows */
+    int32_t S;          /* soft-prompt KV entries, shared by all sequences (0 allowed) */
+    int32_t kv_dtype;   /* CONFU_BF16 | CONFU_F32: type of q, caches, soft KV and out */
+    float   sm_scale;   /* 0 -> D^-1/2 */
+} confu_dims;
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Creates a context on a CUDA device (allocates a small device block for internal
+ * flags).  confu_destroy frees it.  A context is not thread safe. */
+int confu_create(confu_ctx** ctx, int device);
+int confu_destroy(confu_ctx* ctx);
+
+/* Device scratch the attention call needs for these dims (split-KV partial results,
+ * the work plan, the ancestor masks); a pure function of dims and of the device's
+ * SM count.  The caller allocates it and hands it over; it may be shared by all
+ * layers of a step but not by calls that run concurrently. */
+size_t confu_workspace_bytes(const confu_ctx* ctx, const confu_dims* dims);
+int confu_set_workspace(confu_ctx* ctx, void* device_ptr, size_t bytes);
+
+const char* confu_status_string(int code);      /* host return codes and device status codes */
+const char* confu_last_cuda_error(const confu_ctx* ctx);
+
+/* ---- tree attention (Sec. 2, token trees; Sec. 3.1 and Fig. 3) ----------- */
+
+/* Bytes of a caller-held plan buffer for confu_tree_plan. */
+size_t confu_plan_bytes(const confu_ctx* ctx, const confu_dims* dims);
+
+/*
+ * Builds what every layer of one step shares: the ancestor bitmask of each row
+ * (a tree row sees itself and its ancestors; a contemplate row sees itself, its
+ * owner and the owner's ancestors; only contemplate rows see the soft prompts)
+ * and the balanced split-KV work list for this batch's prefix lengths.  Validates
+ * the trees (status codes 1, 2).  All pointers device.  plan: confu_plan_bytes().
+ */
+int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims,
+                    const int64_t* seq_start, const int32_t* prefix_len,
+                    const int32_t* parent,      /* [B][T] */
+                    const int32_t* con_owner,   /* [B][C], may be NULL if C == 0 */
+                    void* plan, int32_t* status, void* stream);
+
+/*
+ * One layer of tree-masked attention.
+ *   out[b][r][h][:] = sum_j softmax_j(sm_scale * q[b][r][h] . k_j) v_j   over the keys row r sees:
+ *   all prefix slots of sequence b, the tree slots its mask allows, and (contemplate
+ *   rows only) the S soft-prompt entries.  KV head of query head h is h / (Hq/Hkv).
+ * q, out: [B][R][Hq][D]; k_cache, v_cache: [n_slots][Hkv][D]; k_soft, v_soft:
+ * [S][Hkv][D] (NULL if S == 0); lse: optional [B][R][Hq] fp32 natural-log softmax
+ * denominators.  plan: a buffer filled by confu_tree_plan for these dims, lengths
+ * and trees, or NULL to have the call build one in the workspace (then parent,
+ * con_owner are read; otherwise they may be NULL).  Accumulation is fp32; bf16
+ * inputs use the tensor-core path when D == 128 and Hq/Hkv <= 4.
+ * Needs the workspace.  All pointers device.
+ */
+int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims,
+                         const void* q, const void* k_cache, const void* v_cache, int64_t n_slots,
+                         const int64_t* seq_start, const int32_t* prefix_len,
+                         const void* k_soft, const void* v_soft,
+                         const int32_t* parent, const int32_t* con_owner,
+                         const void* plan,
+                         void* out, float* lse, int32_t* status, void* stream);
+
+/* ---- acceptance (Sec. 2 steps 3-4; Sec. 3.1 "future prediction associated with the
+ *      last accepted token") ------------------------------------------------ */
+
+/* Device scratch for confu_tree_accept (row statistics). */
+size_t confu_accept_workspace_bytes(int32_t B, int32_t T, int32_t V);
+
+/*
+ * target_logits, draft_logits: [B][T][V] (bf16 or fp32).  Row i of the target is
+ * the distribution of the token after node i; row i of the draft is the one node
+ * i's children were drawn from.  p = softmax(target / temperature), q likewise.
+ * Walk from the root: test the children of the current node in increasing node
+ * index with  u < p(x)/q(x)  (u = uniforms[b][child], x = tokens[b][child]); the
+ * first success is accepted and becomes the current node; a failure replaces p by
+ * norm(max(p - q, 0)) and, with sibling_mode 1 (children drawn without
+ * replacement), removes x from q and renormalises (sibling_mode 0: q unchanged).
+ * When no child is left the next token is drawn from the current p by inverse CDF
+ * in index order with uniforms[b][0]; at a leaf it is drawn from the leaf's target
+ * row.  temperature 0: greedy (accept a child iff its token is the argmax of its
+ * parent's target row, lowest index on ties; deepest such path, lowest node index on
+ * ties; next token = argmax of the last node's row; draft_logits, uniforms unused).
+ * Outputs (device): accept_len [B] (accepted drafts, root excluded); path
+ * [B][CONFU_MAX_DEPTH+1] node ids root first, -1 padded; next_token [B];
+ * future_row [B] = row index in [T,T+C) of the contemplate row owned by the last
+ * accepted node, else by its nearest ancestor that has one, else -1; counters
+ * (optional) [B][4] = ratio tests, rejections, reserved, reserved.
+ * workspace: confu_accept_workspace_bytes().  All pointers device.
+ */
+int confu_tree_accept(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
+                      const void* target_logits, const void* draft_logits,
+                      const int32_t* tokens, const int32_t* parent, const int32_t* con_owner,
+                      const float* uniforms, float temperature, int32_t sibling_mode,
+                      int32_t* accept_len, int32_t* path, int32_t* next_token, int32_t* future_row,
+                      int32_t* counters, void* workspace, size_t workspace_bytes,
+                      int32_t* status, void* stream);
+
+/* ---- KV compaction (Sec. 2 step 4: the accepted sequence is the next input) ---- */
+
+/*
+ * For every layer l < n_layers and for K and V, in place:
+ *   cache[seq_start[b] + P_b + k] = old cache[seq_start[b] + P_b + path[b][k]],  k = 1..accept_len[b]
+ * (P_b = prefix_len[b]; slot P_b, the root, and the prefix stay), and
+ * new_prefix_len[b] = P_b + accept_len[b] + 1.  Slots past the new prefix keep
+ * unspecified contents.  k_cache_layers / v_cache_layers: DEVICE arrays of
+ * n_layers device pointers.  Uses dims->Hkv, D, kv_dtype, B.  All pointers device.
+ */
+int confu_kv_compact(confu_ctx* ctx, const confu_dims* dims, int32_t n_layers,
+                     void* const* k_cache_layers, void* const* v_cache_layers,
+                     const int64_t* seq_start, const int32_t* prefix_len,
+                     const int32_t* accept_len, const int32_t* path,
+                     int32_t* new_prefix_len, int32_t* status, void* stream);
+
+/* ---- writing the step's own K/V into the cache (before confu_tree_attention) ---- */
+
+/*
+ * The verification forward computes K and V of the R query rows themselves (draft tree nodes and
+ * contemplate tokens are processed in one pass, Sec. 3.1); this call places them behind the
+ * prefix: cache[seq_start[b] + prefix_len[b] + r] = rows[b][r], for one layer.
+ * k_rows, v_rows: [B][R][Hkv][D].  All pointers device.
+ */
+int confu_kv_append(confu_ctx* ctx, const confu_dims* dims, const void* k_rows, const void* v_rows,
+                    void* k_cache, void* v_cache, const int64_t* seq_start, const int32_t* prefix_len,
+                    void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONFU_H */

@@ -1,0 +1,535 @@
+// Tree speculative-sampling acceptance.
+//
+//   row_stats_kernel   one streaming pass over every logit row of the target and draft matrices:
+//                      per row chunk the running max, the sum of exp((x - max)/temperature) (online
+//                      softmax), the lowest index of the max, and a non-finite flag.  HBM bound.
+//   accept_walk_kernel one CTA per sequence: the sequential accept / reject walk.  After the k-th
+//                      rejection at a node the target row is norm(max(p - q, 0)) applied k times;
+//                      it is never materialised: each pass re-evaluates the k-level recursion per
+//                      vocabulary entry from the two logit rows (L2 resident) and only the
+//                      normalisers Z_1..Z_k are kept.
+#include <limits.h>
+
+#include "common.cuh"
+
+namespace confu {
+
+constexpr int kStatChunksMax = 16;
+constexpr int kWalkThreads = 512;
+constexpr int kEpt = 8;                                   // vocabulary entries per thread per strip
+constexpr int kStrip = kWalkThreads * kEpt;               // 4096
+constexpr int kMaxStrips = 64;                            // V <= 262144
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct RowStat {
+    float m;        // max raw logit of the chunk
+    float s;        // sum over the chunk of exp((x - m) / temperature)
+    int32_t arg;    // lowest index of the max
+    int32_t flag;   // 1: a non-finite logit was met
+};
+
+size_t accept_workspace_bytes(int B, int T, int /*V*/)
+{
+    return (size_t)2 * B * T * kStatChunksMax * sizeof(RowStat);
+}
+
+template <typename T>
+__device__ __forceinline__ void load8(const T* __restrict__ row, int i0, int V, bool vec_ok, float (&x)[kEpt])
+{
+    if (vec_ok && i0 + kEpt <= V) {
+        if constexpr (sizeof(T) == 2) {
+            const uint4 v = *reinterpret_cast<const uint4*>(row + i0);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                x[2 * j] = __uint_as_float(w[j] << 16);
+                x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+            }
+        } else {
+            const float4 a = *reinterpret_cast<const float4*>(row + i0);
+            const float4 c = *reinterpret_cast<const float4*>(row + i0 + 4);
+            x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+            x[4] = c.x; x[5] = c.y; x[6] = c.z; x[7] = c.w;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < kEpt; ++j) x[j] = (i0 + j < V) ? to_f32(row[i0 + j]) : -INFINITY;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// K3: row statistics
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) row_stats_kernel(const T* __restrict__ tl, const T* __restrict__ dl, int V,
+                                                        int n_rows, int nch, int chunk_elems, float k2,
+                                                        RowStat* __restrict__ stats)
+{
+    const int row = blockIdx.x, chunk = blockIdx.y, mat = blockIdx.z;
+    const T* base = (mat == 0 ? tl : dl) + (size_t)row * V;
+    const bool vec_ok = ((size_t)V * sizeof(T)) % 16 == 0;
+    const int lo = chunk * chunk_elems, hi = min(V, lo + chunk_elems);
+    const int tid = threadIdx.x;
+
+    float m = -INFINITY, s = 0.f, bestv = -INFINITY;
+    int arg = INT_MAX, flag = 0;
+
+    for (int i0 = lo + tid * kEpt; i0 < hi; i0 += 256 * kEpt * 2) {
+        float x[2][kEpt];
+        const int i1 = i0 + 256 * kEpt;
+        load8(base, i0, hi, vec_ok, x[0]);
+        if (i1 < hi) load8(base, i1, hi, vec_ok, x[1]);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int ib = u == 0 ? i0 : i1;
+            if (ib >= hi) break;
+            float lm = x[u][0];
+#pragma unroll
+            for (int j = 1; j < kEpt; ++j) lm = fmaxf(lm, x[u][j]);
+            if (lm > m) { s *= exp2f((m - lm) * k2); m = lm; }
+            float acc = 0.f;
+#pragma unroll
+            for (int j = 0; j < kEpt; ++j) {
+                const float v = x[u][j];
+                const bool in = ib + j < hi;
+                if (in && !(fabsf(v) <= 3.0e38f)) flag = 1;
+                acc += exp2f((v - m) * k2);                      // out-of-range entries are -inf -> 0
+                if (v > bestv) { bestv = v; arg = ib + j; }
+            }
+            s += acc;
+        }
+    }
+    // block reduction of (m, s), (bestv, arg), flag
+    auto merge = [&](float m2, float s2, float v2, int a2, int f2) {
+        const float mm = fmaxf(m, m2);
+        const float c1 = (m == mm) ? 1.f : exp2f((m - mm) * k2);
+        const float c2 = (m2 == mm) ? 1.f : exp2f((m2 - mm) * k2);
+        s = s * c1 + s2 * c2;
+        m = mm;
+        if (v2 > bestv || (v2 == bestv && a2 < arg)) { bestv = v2; arg = a2; }
+        flag |= f2;
+    };
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+        const float s2 = __shfl_xor_sync(0xffffffffu, s, o);
+        const float v2 = __shfl_xor_sync(0xffffffffu, bestv, o);
+        const int a2 = __shfl_xor_sync(0xffffffffu, arg, o);
+        const int f2 = __shfl_xor_sync(0xffffffffu, flag, o);
+        merge(m2, s2, v2, a2, f2);
+    }
+    __shared__ float sm[8], ss[8], sv[8];
+    __shared__ int sa[8], sf[8];
+    if ((tid & 31) == 0) { sm[tid >> 5] = m; ss[tid >> 5] = s; sv[tid >> 5] = bestv; sa[tid >> 5] = arg; sf[tid >> 5] = flag; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 8; ++w) merge(sm[w], ss[w], sv[w], sa[w], sf[w]);
+        RowStat r;
+        r.m = m; r.s = s; r.arg = arg; r.flag = flag;
+        stats[((size_t)mat * n_rows + row) * kStatChunksMax + chunk] = r;
+    }
+    (void)nch;
+}
+
+// ---------------------------------------------------------------------------------------------
+// K4: the walk
+// ---------------------------------------------------------------------------------------------
+struct WalkShared {
+    int code;
+    int cur, len, k, nch, accepted, done, final_level;
+    int path[kPathLen];
+    int ch[kMaxRows];
+    int xs[kMaxRows];          // rejected tokens at the current node
+    float invZ[kMaxRows];      // 1 / Z_j
+    float cs[kMaxRows];        // 1 / (1 - q_{j-1}(x_j))   (sibling_mode 1)
+    float Mt, Md, invZt, invZd;
+    int amax[kMaxRows];
+    double strip[kMaxStrips];
+    double warp_part[kMaxStrips][kWalkThreads / 32];
+    double scan[kWalkThreads / 32];
+    int pick;
+    int pick_last;
+    int tests, rejections;
+    int strip_sel;
+    double strip_off, target;
+};
+
+// merged statistics of one row from its chunk partials (fixed order)
+__device__ inline void merge_row(const RowStat* st, int nch, double inv_temp, float& M, double& Z, int& arg)
+{
+    float mm = -INFINITY;
+    int a = INT_MAX;
+    for (int c = 0; c < nch; ++c)
+        if (st[c].m > mm) { mm = st[c].m; a = st[c].arg; }
+    double z = 0.0;
+    for (int c = 0; c < nch; ++c)
+        if (st[c].m > -INFINITY) z += (double)st[c].s * exp(((double)st[c].m - (double)mm) * inv_temp);
+    M = mm; Z = z; arg = a;
+}
+
+// Weight of vocabulary entry idx after `level` rejections at the current node:
+//   level 0: p_0 = softmax(target)            level k: max(p_{k-1} - q_{k-1}, 0)  (unnormalised p_k)
+__device__ __forceinline__ float weight_at(float tx, float dx, int idx, int level, int mode, const WalkShared& sh,
+                                           float k2)
+{
+    float p = exp2f((tx - sh.Mt) * k2) * sh.invZt;
+    if (level == 0) return p;
+    float q = exp2f((dx - sh.Md) * k2) * sh.invZd;
+    for (int j = 0; j + 1 < level; ++j) {
+        const float pn = fmaxf(p - q, 0.f) * sh.invZ[j];
+        if (mode == 1) q = (idx == sh.xs[j]) ? 0.f : q * sh.cs[j];
+        p = pn;
+    }
+    return fmaxf(p - q, 0.f);
+}
+
+// Sum of weight_at(., level) over the vocabulary, strip by strip, in double; fills sh.strip[].
+template <typename T>
+__device__ double full_pass(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok, int level,
+                            int mode, WalkShared& sh, float k2)
+{
+    const int tid = threadIdx.x, n_strips = (V + kStrip - 1) / kStrip;
+    for (int s0 = 0; s0 < n_strips; s0 += 2) {
+        float tx[2][kEpt], dx[2][kEpt];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i0 = (s0 + u) * kStrip + tid * kEpt;
+            if (s0 + u < n_strips) {
+                load8(trow, i0, V, vec_ok, tx[u]);
+                if (level > 0) load8(drow, i0, V, vec_ok, dx[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (s0 + u >= n_strips) break;
+            const int i0 = (s0 + u) * kStrip + tid * kEpt;
+            double acc = 0.0;
+#pragma unroll
+            for (int j = 0; j < kEpt; ++j)
+                acc += (double)weight_at(tx[u][j], level > 0 ? dx[u][j] : 0.f, i0 + j, level, mode, sh, k2);
+            acc = warp_sum(acc);
+            if ((tid & 31) == 0) sh.warp_part[s0 + u][tid >> 5] = acc;
+        }
+    }
+    __syncthreads();
+    if (tid < n_strips) {
+        double a = 0.0;
+        for (int w = 0; w < kWalkThreads / 32; ++w) a += sh.warp_part[tid][w];
+        sh.strip[tid] = a;
+    }
+    __syncthreads();
+    double tot = 0.0;
+    for (int s = 0; s < n_strips; ++s) tot += sh.strip[s];
+    return tot;
+}
+
+// Inverse CDF in index order over weight_at(., level) using the strip sums of the last full_pass.
+template <typename T>
+__device__ int locate(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok, int level, int mode,
+                      WalkShared& sh, float k2, double u)
+{
+    const int tid = threadIdx.x, n_strips = (V + kStrip - 1) / kStrip;
+    if (tid == 0) {
+        double tot = 0.0;
+        for (int s = 0; s < n_strips; ++s) tot += sh.strip[s];
+        const double target = u * tot;
+        double cum = 0.0;
+        int sel = -1, last_nz = 0;
+        for (int s = 0; s < n_strips; ++s) {
+            if (sh.strip[s] > 0.0) last_nz = s;
+            if (cum + sh.strip[s] > target) { sel = s; break; }
+            cum += sh.strip[s];
+        }
+        if (sel < 0) {                      // rounding left no strip: take the last one that has mass
+            sel = last_nz;
+            cum = 0.0;
+            for (int s = 0; s < sel; ++s) cum += sh.strip[s];
+        }
+        sh.strip_sel = sel; sh.strip_off = cum; sh.target = target;
+        sh.pick = INT_MAX; sh.pick_last = -1;
+    }
+    __syncthreads();
+    const int i0 = sh.strip_sel * kStrip + tid * kEpt;
+    float tx[kEpt], dx[kEpt];
+    load8(trow, i0, V, vec_ok, tx);
+    if (level > 0) load8(drow, i0, V, vec_ok, dx);
+    float w[kEpt];
+    double loc = 0.0;
+#pragma unroll
+    for (int j = 0; j < kEpt; ++j) {
+        w[j] = weight_at(tx[j], level > 0 ? dx[j] : 0.f, i0 + j, level, mode, sh, k2);
+        loc += (double)w[j];
+    }
+    // block exclusive scan of loc (double): warp scan + warp totals
+    double incl = loc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((tid & 31) >= o) incl += t;
+    }
+    if ((tid & 31) == 31) sh.scan[tid >> 5] = incl;
+    __syncthreads();
+    double off = sh.strip_off;
+    for (int wi = 0; wi < (tid >> 5); ++wi) off += sh.scan[wi];
+    double run = off + (incl - loc);
+    int cand = INT_MAX, last = -1;
+#pragma unroll
+    for (int j = 0; j < kEpt; ++j) {
+        run += (double)w[j];
+        if (w[j] > 0.f) last = i0 + j;
+        if (cand == INT_MAX && run > sh.target) cand = i0 + j;
+    }
+    if (cand != INT_MAX) atomicMin(&sh.pick, cand);
+    if (last >= 0) atomicMax(&sh.pick_last, last);
+    __syncthreads();
+    int res = sh.pick != INT_MAX ? sh.pick : (sh.pick_last >= 0 ? sh.pick_last : 0);
+    __syncthreads();
+    return res;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
+    int Tn, int C, int V, const T* __restrict__ tl, const T* __restrict__ dl, const int32_t* __restrict__ tokens,
+    const int32_t* __restrict__ parent, const int32_t* __restrict__ con_owner, const float* __restrict__ uniforms,
+    float temperature, int mode, int nch, int n_rows, const RowStat* __restrict__ stats,
+    int32_t* __restrict__ accept_len, int32_t* __restrict__ path, int32_t* __restrict__ next_token,
+    int32_t* __restrict__ future_row, int32_t* __restrict__ counters, int32_t* __restrict__ status)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    WalkShared& sh = *reinterpret_cast<WalkShared*>(smem_raw);
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int32_t* par = parent + (size_t)b * Tn;
+    const int32_t* tok = tokens + (size_t)b * Tn;
+    const int32_t* own = con_owner ? con_owner + (size_t)b * C : nullptr;
+    const bool greedy = !(temperature > 0.f);
+    const RowStat* st_t = stats + ((size_t)0 * n_rows + (size_t)b * Tn) * kStatChunksMax;
+    const RowStat* st_d = stats + ((size_t)1 * n_rows + (size_t)b * Tn) * kStatChunksMax;
+    const bool vec_ok = ((size_t)V * sizeof(T)) % 16 == 0;
+
+    if (tid == 0) sh.code = INT_MAX;
+    __syncthreads();
+    // ---- validation (lowest code wins, like a sequential check in code order) ----
+    if (tid < Tn) {
+        int code = INT_MAX;
+        const int p = par[tid];
+        if (tid == 0 ? (p != -1) : (p < 0 || p >= tid)) code = CONFU_ST_BAD_PARENT;
+        else if (tok[tid] < 0 || tok[tid] >= V) code = CONFU_ST_BAD_TOKEN;
+        else {
+            if (!greedy && mode == 1 && tid > 0)
+                for (int j = tid + 1; j < Tn; ++j)
+                    if (par[j] == p && tok[j] == tok[tid]) code = CONFU_ST_DUP_SIBLING;
+            if (code == INT_MAX)
+                for (int c = 0; c < nch; ++c)
+                    if (st_t[(size_t)tid * kStatChunksMax + c].flag ||
+                        (!greedy && st_d[(size_t)tid * kStatChunksMax + c].flag))
+                        code = CONFU_ST_NONFINITE;
+        }
+        if (code != INT_MAX) atomicMin(&sh.code, code);
+    }
+    if (tid < C) {
+        const int o = own[tid];
+        if (o < 0 || o >= Tn) atomicMin(&sh.code, (int)CONFU_ST_BAD_OWNER);
+    }
+    __syncthreads();
+    int32_t* pth = path + (size_t)b * kPathLen;
+    if (sh.code != INT_MAX) {
+        if (tid < kPathLen) pth[tid] = tid == 0 ? 0 : -1;
+        if (tid == 0) {
+            accept_len[b] = 0; next_token[b] = -1;
+            if (future_row) future_row[b] = -1;
+            if (counters) { counters[4 * b] = 0; counters[4 * b + 1] = 0; counters[4 * b + 2] = 0; counters[4 * b + 3] = 0; }
+            if (status) status[b] = sh.code;
+        }
+        return;
+    }
+    const double inv_temp = greedy ? 1.0 : 1.0 / (double)temperature;
+    const float k2 = (float)inv_temp * kLog2e;
+
+    if (tid == 0) { sh.cur = 0; sh.len = 0; sh.path[0] = 0; sh.tests = 0; sh.rejections = 0; sh.done = 0; }
+
+    if (greedy) {
+        if (tid < Tn) {
+            float M; double Z; int a;
+            merge_row(st_t + (size_t)tid * kStatChunksMax, nch, 1.0, M, Z, a);
+            sh.amax[tid] = a;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            unsigned long long keep = 1ull;
+            int depth[kMaxRows];
+            depth[0] = 0;
+            int best = 0;
+            for (int i = 1; i < Tn; ++i) {
+                const int pa = par[i];
+                depth[i] = depth[pa] + 1;
+                if (!((keep >> pa) & 1ull)) continue;
+                if (tok[i] == sh.amax[pa]) {
+                    keep |= 1ull << i;
+                    if (depth[i] > depth[best]) best = i;
+                }
+            }
+            sh.len = depth[best];
+            for (int a = best, k = sh.len; a >= 0; a = par[a], --k) sh.path[k] = a;
+            sh.cur = best;
+            next_token[b] = sh.amax[best];
+        }
+        __syncthreads();
+    } else {
+        const double u0 = (double)uniforms[(size_t)b * Tn];
+        for (;;) {
+            // ---- set up the current node ----
+            if (tid == 0) {
+                const int cur = sh.cur;
+                float M; double Z; int a;
+                merge_row(st_t + (size_t)cur * kStatChunksMax, nch, inv_temp, M, Z, a);
+                sh.Mt = M; sh.invZt = (float)(1.0 / Z);
+                merge_row(st_d + (size_t)cur * kStatChunksMax, nch, inv_temp, M, Z, a);
+                sh.Md = M; sh.invZd = (float)(1.0 / Z);
+                int n = 0;
+                for (int i = cur + 1; i < Tn; ++i) if (par[i] == cur) sh.ch[n++] = i;
+                sh.nch = n; sh.k = 0; sh.accepted = -1;
+            }
+            __syncthreads();
+            const int cur = sh.cur;
+            const T* trow = tl + ((size_t)b * Tn + cur) * V;
+            const T* drow = dl + ((size_t)b * Tn + cur) * V;
+            int final_level = 0;
+            bool have_strips = false;
+            for (int ci = 0; ci < sh.nch; ++ci) {
+                const int c = sh.ch[ci];
+                // ---- ratio test of child c (thread 0, double) ----
+                if (tid == 0) {
+                    const int x = tok[c];
+                    const double u = (double)uniforms[(size_t)b * Tn + c];
+                    double p = exp(((double)to_f32(trow[x]) - (double)sh.Mt) * inv_temp) * (double)sh.invZt;
+                    double q = exp(((double)to_f32(drow[x]) - (double)sh.Md) * inv_temp) * (double)sh.invZd;
+                    for (int j = 0; j < sh.k; ++j) {
+                        const double pn = fmax(p - q, 0.0) * (double)sh.invZ[j];
+                        if (mode == 1) q = (x == sh.xs[j]) ? 0.0 : q * (double)sh.cs[j];
+                        p = pn;
+                    }
+                    const double ratio = (q == 0.0) ? (p > 0.0 ? INFINITY : 0.0) : p / q;
+                    ++sh.tests;
+                    if (u < ratio) sh.accepted = c;
+                    else {
+                        ++sh.rejections;
+                        sh.xs[sh.k] = x;
+                        const double rem = 1.0 - q;
+                        sh.cs[sh.k] = rem > 0.0 ? (float)(1.0 / rem) : 0.f;
+                        sh.done = (mode == 1 && !(rem > 0.0)) ? 1 : 0;      // q has no mass left: stop testing
+                    }
+                }
+                __syncthreads();
+                if (sh.accepted >= 0) break;
+                // ---- rejection k+1: normaliser of the new residual ----
+                const int level = sh.k + 1;
+                const double Z = full_pass(trow, drow, V, vec_ok, level, mode, sh, k2);
+                have_strips = true;
+                final_level = level;
+                if (tid == 0) {
+                    if (Z > 0.0) { sh.invZ[sh.k] = (float)(1.0 / Z); sh.k = level; }
+                    else { sh.done = 2; }                                    // no mass: fall back to the target row
+                }
+                __syncthreads();
+                if (sh.done) break;
+            }
+            if (sh.accepted >= 0) {
+                __syncthreads();
+                if (tid == 0) {
+                    if (sh.len + 1 > CONFU_MAX_DEPTH) sh.done = 3;
+                    else { sh.path[++sh.len] = sh.accepted; sh.cur = sh.accepted; }
+                }
+                __syncthreads();
+                if (sh.done == 3) break;
+                continue;
+            }
+            // ---- final draw at this node ----
+            if (sh.done == 2) { final_level = 0; have_strips = false; }
+            if (!have_strips) full_pass(trow, drow, V, vec_ok, final_level, mode, sh, k2);
+            const int pick = locate(trow, drow, V, vec_ok, final_level, mode, sh, k2, u0);
+            if (tid == 0) next_token[b] = pick;
+            break;
+        }
+        __syncthreads();
+        if (sh.done == 3) {              // path buffer exhausted
+            if (tid < kPathLen) pth[tid] = tid == 0 ? 0 : -1;
+            if (tid == 0) {
+                accept_len[b] = 0; next_token[b] = -1;
+                if (future_row) future_row[b] = -1;
+                if (status) status[b] = CONFU_ST_TOO_DEEP;
+            }
+            return;
+        }
+        if (sh.done == 2 && tid == 0 && status) status[b] = CONFU_ST_DEGENERATE;
+    }
+    // ---- outputs ----
+    if (tid < kPathLen) pth[tid] = tid <= sh.len ? sh.path[tid] : -1;
+    if (tid == 0) {
+        accept_len[b] = sh.len;
+        if (future_row) {
+            int fr = -1;
+            for (int a = sh.cur; a >= 0 && fr < 0; a = par[a])
+                for (int k = 0; k < C; ++k)
+                    if (own[k] == a) { fr = Tn + k; break; }
+            future_row[b] = fr;
+        }
+        if (counters) {
+            counters[4 * b] = sh.tests; counters[4 * b + 1] = sh.rejections;
+            counters[4 * b + 2] = 0; counters[4 * b + 3] = 0;
+        }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, const void* dl, const int32_t* tokens,
+                                   const int32_t* parent, const int32_t* con_owner, const float* uniforms,
+                                   float temperature, int mode, int32_t* accept_len, int32_t* path,
+                                   int32_t* next_token, int32_t* future_row, int32_t* counters, void* workspace,
+                                   int32_t* status, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    const bool greedy = !(temperature > 0.f);
+    const int n_rows = B * Tn;
+    const int nmat = greedy ? 1 : 2;
+    // enough CTAs to fill the machine a few times over, chunks a multiple of the vector width
+    int nch = (148 * 8 + n_rows * nmat - 1) / (n_rows * nmat);
+    nch = nch < 1 ? 1 : (nch > kStatChunksMax ? kStatChunksMax : nch);
+    int chunk_elems = (V + nch - 1) / nch;
+    chunk_elems = (chunk_elems + 15) / 16 * 16;
+    nch = (V + chunk_elems - 1) / chunk_elems;
+    const float k2 = (greedy ? 1.f : 1.f / temperature) * kLog2e;
+    RowStat* stats = (RowStat*)workspace;
+    row_stats_kernel<T><<<dim3(n_rows, nch, nmat), 256, 0, st>>>((const T*)tl, (const T*)dl, V, n_rows, nch,
+                                                                 chunk_elems, k2, stats);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t smem = sizeof(WalkShared);
+    static bool attr_done[2] = {false, false};
+    const int ti = sizeof(T) == 2 ? 0 : 1;
+    if (!attr_done[ti]) {
+        e = cudaFuncSetAttribute(accept_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done[ti] = true;
+    }
+    accept_walk_kernel<T><<<B, kWalkThreads, smem, st>>>(Tn, C, V, (const T*)tl, (const T*)dl, tokens, parent,
+                                                         con_owner, uniforms, temperature, mode, nch, n_rows, stats,
+                                                         accept_len, path, next_token, future_row, counters, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_accept(const Ctx*, int B, int T, int C, int V, int logit_dtype, const void* tl, const void* dl,
+                          const int32_t* tokens, const int32_t* parent, const int32_t* con_owner,
+                          const float* uniforms, float temperature, int sibling_mode, int32_t* accept_len,
+                          int32_t* path, int32_t* next_token, int32_t* future_row, int32_t* counters,
+                          void* workspace, int32_t* status, cudaStream_t st)
+{
+    if (logit_dtype == CONFU_F32)
+        return launch_accept_t<float>(B, T, C, V, tl, dl, tokens, parent, con_owner, uniforms, temperature,
+                                      sibling_mode, accept_len, path, next_token, future_row, counters, workspace,
+                                      status, st);
+    return launch_accept_t<__nv_bfloat16>(B, T, C, V, tl, dl, tokens, parent, con_owner, uniforms, temperature,
+                                          sibling_mode, accept_len, path, next_token, future_row, counters, workspace,
+                                          status, st);
+}
+
+}  // namespace confu

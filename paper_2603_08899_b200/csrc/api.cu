@@ -1,0 +1,243 @@
+// C ABI of the library: argument checks, workspace carving, kernel launches.
+#include <new>
+
+#include "common.cuh"
+
+using namespace confu;
+
+struct confu_ctx : public confu::Ctx {};
+
+namespace {
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+int check_dims(const confu_dims* d)
+{
+    if (!d) return CONFU_ERR_ARG;
+    if (d->B < 0 || d->Hq <= 0 || d->Hkv <= 0 || d->T <= 0 || d->C < 0 || d->S < 0) return CONFU_ERR_SHAPE;
+    if (d->Hq % d->Hkv != 0) return CONFU_ERR_SHAPE;
+    if (d->D != 64 && d->D != 128) return CONFU_ERR_SHAPE;
+    if (d->kv_dtype != CONFU_BF16 && d->kv_dtype != CONFU_F32) return CONFU_ERR_ARG;
+    if (d->T + d->C > CONFU_MAX_ROWS) return CONFU_ERR_UNSUPPORTED;
+    if (!(d->sm_scale >= 0.f)) return CONFU_ERR_ARG;
+    return CONFU_OK;
+}
+
+int cuda_fail(confu_ctx* ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_error = e;
+    return CONFU_ERR_CUDA;
+}
+
+// workspace carving: [plan built by the attention call itself][split-KV partial slots]
+size_t ws_plan_offset() { return 0; }
+size_t ws_partial_offset(const confu_dims* d) { return align_up(plan_bytes(d->B), 256); }
+size_t ws_total(const confu_ctx* ctx, const confu_dims* d)
+{
+    return ws_partial_offset(d) + (size_t)2 * ctx->sm_count * partial_slot_bytes();
+}
+
+}  // namespace
+
+namespace confu {
+bool tc_attention_supported(const confu_dims& d);
+cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
+                                const void* v_cache, int64_t n_slots, const int64_t* seq_start,
+                                const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
+                                void* partials, void* out, float* lse, int32_t* status, cudaStream_t st);
+}  // namespace confu
+
+extern "C" {
+
+int confu_create(confu_ctx** out, int device)
+{
+    if (!out) return CONFU_ERR_ARG;
+    *out = nullptr;
+    confu_ctx* c = new (std::nothrow) confu_ctx();
+    if (!c) return CONFU_ERR_ARG;
+    c->device = device;
+    c->workspace = nullptr;
+    c->workspace_bytes = 0;
+    c->dev_flags = nullptr;
+    c->last_error = cudaSuccess;
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&c->dev_flags, 256);
+    if (e == cudaSuccess) e = cudaMemset(c->dev_flags, 0, 256);
+    if (e != cudaSuccess) {
+        delete c;
+        return CONFU_ERR_CUDA;
+    }
+    *out = c;
+    return CONFU_OK;
+}
+
+int confu_destroy(confu_ctx* ctx)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    if (ctx->dev_flags) cudaFree(ctx->dev_flags);
+    delete ctx;
+    return CONFU_OK;
+}
+
+size_t confu_workspace_bytes(const confu_ctx* ctx, const confu_dims* dims)
+{
+    if (!ctx || check_dims(dims) != CONFU_OK) return 0;
+    return ws_total(ctx, dims);
+}
+
+int confu_set_workspace(confu_ctx* ctx, void* device_ptr, size_t bytes)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    if (device_ptr && misaligned(device_ptr)) return CONFU_ERR_ALIGN;
+    ctx->workspace = device_ptr;
+    ctx->workspace_bytes = device_ptr ? bytes : 0;
+    return CONFU_OK;
+}
+
+const char* confu_status_string(int code)
+{
+    switch (code) {
+        case CONFU_OK: return "ok";
+        case CONFU_ERR_ARG: return "bad argument";
+        case CONFU_ERR_SHAPE: return "unsupported or inconsistent shape";
+        case CONFU_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case CONFU_ERR_WORKSPACE: return "workspace missing or too small";
+        case CONFU_ERR_UNSUPPORTED: return "configuration not supported";
+        case CONFU_ERR_CUDA: return "CUDA call failed";
+        case CONFU_ST_BAD_PARENT: return "malformed tree: parent index";
+        case CONFU_ST_BAD_OWNER: return "malformed tree: contemplate owner";
+        case CONFU_ST_BAD_TOKEN: return "token id out of range";
+        case CONFU_ST_DUP_SIBLING: return "duplicate sibling tokens";
+        case CONFU_ST_NONFINITE: return "non-finite logit";
+        case CONFU_ST_TIMEOUT: return "bounded device wait expired";
+        case CONFU_ST_DEGENERATE: return "residual distribution without mass";
+        case CONFU_ST_TOO_DEEP: return "accepted path longer than CONFU_MAX_DEPTH";
+        default: return "unknown code";
+    }
+}
+
+const char* confu_last_cuda_error(const confu_ctx* ctx)
+{
+    return cudaGetErrorString(ctx ? ctx->last_error : cudaSuccess);
+}
+
+size_t confu_plan_bytes(const confu_ctx* ctx, const confu_dims* dims)
+{
+    if (!ctx || check_dims(dims) != CONFU_OK) return 0;
+    return plan_bytes(dims->B);
+}
+
+int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims, const int64_t* seq_start, const int32_t* prefix_len,
+                    const int32_t* parent, const int32_t* con_owner, void* plan, int32_t* status, void* stream)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    int rc = check_dims(dims);
+    if (rc != CONFU_OK) return rc;
+    if (!plan) return CONFU_ERR_ARG;
+    if (dims->B > 0 && (!seq_start || !prefix_len || !parent || (dims->C > 0 && !con_owner))) return CONFU_ERR_ARG;
+    if (misaligned(plan)) return CONFU_ERR_ALIGN;
+    cudaError_t e = launch_plan(ctx, *dims, seq_start, prefix_len, parent, con_owner, plan, status, (cudaStream_t)stream);
+    return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
+}
+
+int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims, const void* q, const void* k_cache,
+                         const void* v_cache, int64_t n_slots, const int64_t* seq_start, const int32_t* prefix_len,
+                         const void* k_soft, const void* v_soft, const int32_t* parent, const int32_t* con_owner,
+                         const void* plan, void* out, float* lse, int32_t* status, void* stream)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    int rc = check_dims(dims);
+    if (rc != CONFU_OK) return rc;
+    if (dims->B == 0) return CONFU_OK;
+    if (!q || !k_cache || !v_cache || !seq_start || !prefix_len || !out || n_slots <= 0) return CONFU_ERR_ARG;
+    if (dims->S > 0 && (!k_soft || !v_soft)) return CONFU_ERR_ARG;
+    if (!plan && (!parent || (dims->C > 0 && !con_owner))) return CONFU_ERR_ARG;
+    if (misaligned(q) || misaligned(k_cache) || misaligned(v_cache) || misaligned(out) || misaligned(k_soft) ||
+        misaligned(v_soft) || misaligned(plan))
+        return CONFU_ERR_ALIGN;
+    if (!ctx->workspace || ctx->workspace_bytes < ws_total(ctx, dims)) return CONFU_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* ws = (char*)ctx->workspace;
+    const void* use_plan = plan;
+    if (!plan) {
+        void* own_plan = ws + ws_plan_offset();
+        cudaError_t e = launch_plan(ctx, *dims, seq_start, prefix_len, parent, con_owner, own_plan, status, st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        use_plan = own_plan;
+    }
+    cudaError_t e;
+    if (tc_attention_supported(*dims))
+        e = launch_attention_tc(ctx, *dims, q, k_cache, v_cache, n_slots, seq_start, prefix_len, k_soft, v_soft,
+                                use_plan, ws + ws_partial_offset(dims), out, lse, status, st);
+    else
+        e = launch_attention_generic(ctx, *dims, q, k_cache, v_cache, seq_start, prefix_len, k_soft, v_soft, use_plan,
+                                     out, lse, st);
+    return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
+}
+
+size_t confu_accept_workspace_bytes(int32_t B, int32_t T, int32_t V)
+{
+    if (B < 0 || T <= 0 || V <= 0) return 0;
+    return accept_workspace_bytes(B, T, V);
+}
+
+int confu_tree_accept(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
+                      const void* target_logits, const void* draft_logits, const int32_t* tokens,
+                      const int32_t* parent, const int32_t* con_owner, const float* uniforms, float temperature,
+                      int32_t sibling_mode, int32_t* accept_len, int32_t* path, int32_t* next_token,
+                      int32_t* future_row, int32_t* counters, void* workspace, size_t workspace_bytes,
+                      int32_t* status, void* stream)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    if (B < 0 || T <= 0 || C < 0 || V <= 0) return CONFU_ERR_SHAPE;
+    if (logit_dtype != CONFU_BF16 && logit_dtype != CONFU_F32) return CONFU_ERR_ARG;
+    if (sibling_mode != 0 && sibling_mode != 1) return CONFU_ERR_ARG;
+    if (!(temperature >= 0.f)) return CONFU_ERR_ARG;
+    if (T > CONFU_MAX_ROWS || C > CONFU_MAX_ROWS || V > 262144) return CONFU_ERR_UNSUPPORTED;
+    if (B == 0) return CONFU_OK;
+    if (!target_logits || !tokens || !parent || !accept_len || !path || !next_token) return CONFU_ERR_ARG;
+    if (C > 0 && !con_owner) return CONFU_ERR_ARG;
+    if (temperature > 0.f && (!draft_logits || !uniforms)) return CONFU_ERR_ARG;
+    if (misaligned(target_logits) || misaligned(draft_logits) || misaligned(workspace)) return CONFU_ERR_ALIGN;
+    if (!workspace || workspace_bytes < accept_workspace_bytes(B, T, V)) return CONFU_ERR_WORKSPACE;
+    cudaError_t e = launch_accept(ctx, B, T, C, V, logit_dtype, target_logits, draft_logits, tokens, parent, con_owner,
+                                  uniforms, temperature, sibling_mode, accept_len, path, next_token, future_row,
+                                  counters, workspace, status, (cudaStream_t)stream);
+    return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
+}
+
+int confu_kv_compact(confu_ctx* ctx, const confu_dims* dims, int32_t n_layers, void* const* k_cache_layers,
+                     void* const* v_cache_layers, const int64_t* seq_start, const int32_t* prefix_len,
+                     const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len, int32_t* status,
+                     void* stream)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    int rc = check_dims(dims);
+    if (rc != CONFU_OK) return rc;
+    if (n_layers < 0) return CONFU_ERR_ARG;
+    if (dims->B == 0) return CONFU_OK;
+    if (!seq_start || !prefix_len || !accept_len || !path) return CONFU_ERR_ARG;
+    if (n_layers > 0 && (!k_cache_layers || !v_cache_layers)) return CONFU_ERR_ARG;
+    const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : 4);
+    cudaError_t e = launch_compact(ctx, dims->B, n_layers, row_bytes, k_cache_layers, v_cache_layers, seq_start,
+                                   prefix_len, accept_len, path, new_prefix_len, status, (cudaStream_t)stream);
+    return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
+}
+
+int confu_kv_append(confu_ctx* ctx, const confu_dims* dims, const void* k_rows, const void* v_rows, void* k_cache,
+                    void* v_cache, const int64_t* seq_start, const int32_t* prefix_len, void* stream)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    int rc = check_dims(dims);
+    if (rc != CONFU_OK) return rc;
+    if (dims->B == 0) return CONFU_OK;
+    if (!k_rows || !v_rows || !k_cache || !v_cache || !seq_start || !prefix_len) return CONFU_ERR_ARG;
+    if (misaligned(k_rows) || misaligned(v_rows) || misaligned(k_cache) || misaligned(v_cache)) return CONFU_ERR_ALIGN;
+    const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : 4);
+    cudaError_t e = launch_append(dims->B, dims->T + dims->C, row_bytes, k_rows, v_rows, k_cache, v_cache, seq_start,
+                                  prefix_len, (cudaStream_t)stream);
+    return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
+}
+
+}  // extern "C"

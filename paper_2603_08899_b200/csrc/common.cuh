@@ -1,0 +1,137 @@
+// Shared declarations of the CUDA library (not used by the CPU oracle).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "confu.h"
+
+namespace confu {
+
+constexpr int kMaxRows = CONFU_MAX_ROWS;        // R = T + C <= 64: one 64-bit mask word per row
+constexpr int kPathLen = CONFU_MAX_DEPTH + 1;
+constexpr int kTileKeys = 128;                  // keys per attention tile (tensor-core path)
+
+// ---------------------------------------------------------------------------
+// Plan buffer (device).  Built once per step by plan_kernel, read by every layer.
+//   PlanHeader
+//   uint64 mask[B][64]        bit j of mask[b][r]: row r sees tree slot j
+//   int32  bad[B]             non-zero: malformed tree, sequence skipped
+//   int32  tiles[B]           key tiles of one (sequence, kv head) pair, soft-prompt tile included
+//   int64  tile_base[B + 1]   flat index of the first tile of sequence b (all Hkv heads), exclusive scan
+// ---------------------------------------------------------------------------
+struct PlanHeader {
+    int32_t B, Hkv, T, C, S, R;
+    int32_t n_ctas;            // CTAs of the tensor-core attention launch (<= SM count)
+    int32_t pad;
+    int64_t n_tiles;           // total tiles over all (sequence, kv head) pairs
+};
+
+struct PlanView {
+    PlanHeader* hdr;
+    uint64_t* mask;
+    int32_t* bad;
+    int32_t* tiles;
+    int64_t* tile_base;
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+__host__ __device__ inline size_t plan_bytes(int B)
+{
+    size_t n = align_up(sizeof(PlanHeader), 256);
+    n += align_up((size_t)B * kMaxRows * sizeof(uint64_t), 256);
+    n += align_up((size_t)B * sizeof(int32_t), 256);
+    n += align_up((size_t)B * sizeof(int32_t), 256);
+    n += align_up((size_t)(B + 1) * sizeof(int64_t), 256);
+    return n;
+}
+
+__host__ __device__ inline PlanView plan_view(void* base, int B)
+{
+    char* p = (char*)base;
+    PlanView v;
+    v.hdr = (PlanHeader*)p;                  p += align_up(sizeof(PlanHeader), 256);
+    v.mask = (uint64_t*)p;                   p += align_up((size_t)B * kMaxRows * sizeof(uint64_t), 256);
+    v.bad = (int32_t*)p;                     p += align_up((size_t)B * sizeof(int32_t), 256);
+    v.tiles = (int32_t*)p;                   p += align_up((size_t)B * sizeof(int32_t), 256);
+    v.tile_base = (int64_t*)p;
+    return v;
+}
+
+// Split-KV partial of the tensor-core path: per CTA two slots of M_MAX rows x (D fp32 + max + sum).
+constexpr int kPartRows = 256;                  // 2 M-tiles of 128 rows
+constexpr int kPartD = 128;
+__host__ __device__ inline size_t partial_slot_bytes()
+{
+    return (size_t)kPartRows * kPartD * sizeof(float) + (size_t)kPartRows * 2 * sizeof(float);
+}
+
+struct Ctx {
+    int device;
+    int sm_count;
+    void* workspace;
+    size_t workspace_bytes;
+    int32_t* dev_flags;        // small device block owned by the context
+    cudaError_t last_error;
+};
+
+// ---------------------------------------------------------------------------
+// element access
+// ---------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---------------------------------------------------------------------------
+// launchers (defined in the .cu files)
+// ---------------------------------------------------------------------------
+cudaError_t launch_plan(const Ctx* ctx, const confu_dims& d, const int64_t* seq_start, const int32_t* prefix_len,
+                        const int32_t* parent, const int32_t* con_owner, void* plan, int32_t* status,
+                        cudaStream_t st);
+
+cudaError_t launch_attention_generic(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
+                                     const void* v_cache, const int64_t* seq_start, const int32_t* prefix_len,
+                                     const void* k_soft, const void* v_soft, const void* plan, void* out,
+                                     float* lse, cudaStream_t st);
+
+cudaError_t launch_accept(const Ctx* ctx, int B, int T, int C, int V, int logit_dtype, const void* tl,
+                          const void* dl, const int32_t* tokens, const int32_t* parent, const int32_t* con_owner,
+                          const float* uniforms, float temperature, int sibling_mode, int32_t* accept_len,
+                          int32_t* path, int32_t* next_token, int32_t* future_row, int32_t* counters,
+                          void* workspace, int32_t* status, cudaStream_t st);
+size_t accept_workspace_bytes(int B, int T, int V);
+
+cudaError_t launch_compact(const Ctx* ctx, int B, int n_layers, int64_t row_bytes, void* const* k_layers,
+                           void* const* v_layers, const int64_t* seq_start, const int32_t* prefix_len,
+                           const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len,
+                           int32_t* status, cudaStream_t st);
+
+cudaError_t launch_append(int B, int R, int64_t row_bytes, const void* k_rows, const void* v_rows, void* k_cache,
+                          void* v_cache, const int64_t* seq_start, const int32_t* prefix_len, cudaStream_t st);
+
+}  // namespace confu

@@ -1,0 +1,86 @@
+// KV compaction of the accepted path: cache[P + k] <- cache[P + path[k]], k = 1..accept_len, for
+// every layer and for K and V, in place.
+//
+// In-place safety without a snapshot: node ids are topologically numbered (parent < child), so
+// path[k] >= k, the sources path[1] < path[2] < ... are increasing, and destination k can only
+// coincide with a source of an EARLIER step (path[j] = k needs j <= k).  Each thread owns one
+// 16-byte column of the row and walks k upwards in batches (all loads of a batch before its
+// stores), so within a thread every source is read before any step at or after it overwrites
+// that slot, and different threads never touch each other's columns.
+#include "common.cuh"
+
+namespace confu {
+
+constexpr int kCompactBatch = 8;
+
+__global__ void __launch_bounds__(128) compact_kernel(int n_layers, int64_t row_vecs, void* const* __restrict__ k_layers,
+                                                      void* const* __restrict__ v_layers,
+                                                      const int64_t* __restrict__ seq_start,
+                                                      const int32_t* __restrict__ prefix_len,
+                                                      const int32_t* __restrict__ accept_len,
+                                                      const int32_t* __restrict__ path,
+                                                      int32_t* __restrict__ new_prefix_len)
+{
+    const int b = blockIdx.z, layer = blockIdx.y >> 1, kv = blockIdx.y & 1;
+    const int64_t col = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int a = accept_len[b];
+    a = a < 0 ? 0 : (a > CONFU_MAX_DEPTH ? CONFU_MAX_DEPTH : a);
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && new_prefix_len)
+        new_prefix_len[b] = prefix_len[b] + a + 1;
+    if (a == 0 || col >= row_vecs) return;
+    uint4* pool = reinterpret_cast<uint4*>(kv ? v_layers[layer] : k_layers[layer]);
+    const int64_t root = seq_start[b] + prefix_len[b];
+    const int32_t* pth = path + (size_t)b * kPathLen;
+    for (int k0 = 1; k0 <= a; k0 += kCompactBatch) {
+        uint4 buf[kCompactBatch];
+#pragma unroll
+        for (int j = 0; j < kCompactBatch; ++j)
+            if (k0 + j <= a) buf[j] = pool[(root + pth[k0 + j]) * row_vecs + col];
+#pragma unroll
+        for (int j = 0; j < kCompactBatch; ++j)
+            if (k0 + j <= a) pool[(root + k0 + j) * row_vecs + col] = buf[j];
+    }
+    (void)n_layers;
+}
+
+// cache[seq_start[b] + prefix_len[b] + r] = rows[b][r]  (K and V of the step's own query rows)
+__global__ void __launch_bounds__(128) append_kernel(int R, int64_t row_vecs, const uint4* __restrict__ k_rows,
+                                                     const uint4* __restrict__ v_rows, uint4* __restrict__ k_cache,
+                                                     uint4* __restrict__ v_cache, const int64_t* __restrict__ seq_start,
+                                                     const int32_t* __restrict__ prefix_len)
+{
+    const int r = blockIdx.x, b = blockIdx.y, kv = blockIdx.z;
+    const uint4* src = (kv ? v_rows : k_rows) + ((size_t)b * R + r) * row_vecs;
+    uint4* dst = (kv ? v_cache : k_cache) + (size_t)(seq_start[b] + prefix_len[b] + r) * row_vecs;
+    for (int64_t c = threadIdx.x; c < row_vecs; c += blockDim.x) dst[c] = src[c];
+}
+
+cudaError_t launch_append(int B, int R, int64_t row_bytes, const void* k_rows, const void* v_rows, void* k_cache,
+                          void* v_cache, const int64_t* seq_start, const int32_t* prefix_len, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    append_kernel<<<dim3(R, B, 2), 128, 0, st>>>(R, row_bytes / 16, (const uint4*)k_rows, (const uint4*)v_rows,
+                                                 (uint4*)k_cache, (uint4*)v_cache, seq_start, prefix_len);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compact(const Ctx*, int B, int n_layers, int64_t row_bytes, void* const* k_layers,
+                           void* const* v_layers, const int64_t* seq_start, const int32_t* prefix_len,
+                           const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len,
+                           int32_t* /*status*/, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    const int64_t row_vecs = row_bytes / 16;
+    // with no layers there is still new_prefix_len to write: one block row does it
+    dim3 grid((unsigned)((row_vecs + 127) / 128), (unsigned)(n_layers > 0 ? 2 * n_layers : 1), (unsigned)B);
+    if (n_layers == 0) {
+        compact_kernel<<<dim3(1, 1, B), 128, 0, st>>>(0, 0, k_layers, v_layers, seq_start, prefix_len, accept_len, path,
+                                                       new_prefix_len);
+    } else {
+        compact_kernel<<<grid, 128, 0, st>>>(n_layers, row_vecs, k_layers, v_layers, seq_start, prefix_len, accept_len,
+                                             path, new_prefix_len);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace confu

@@ -1,0 +1,98 @@
+// Step-level planning kernel: tree validation, ancestor bitmasks, split-KV tile counts.
+//
+// Mask rule (tree attention over a token tree, with one contemplate token hung on a node's
+// branch): a tree row sees itself and its ancestors; a contemplate row sees itself, its owner
+// and the owner's ancestors.  Bit j of mask[b][r] says "row r sees tree slot j".
+#include "common.cuh"
+
+namespace confu {
+
+__global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, const int64_t* __restrict__ seq_start,
+                                                   const int32_t* __restrict__ prefix_len,
+                                                   const int32_t* __restrict__ parent,
+                                                   const int32_t* __restrict__ con_owner, void* plan_raw,
+                                                   int32_t* status)
+{
+    const int B = d.B, T = d.T, C = d.C, R = d.T + d.C;
+    PlanView pv = plan_view(plan_raw, B);
+    __shared__ int s_bad[4];
+    __shared__ uint64_t s_mask[4][kMaxRows];
+    const int grp = threadIdx.x >> 6, r = threadIdx.x & 63;
+
+    for (int b0 = 0; b0 < B; b0 += 4) {
+        const int b = b0 + grp;
+        if (r == 0) s_bad[grp] = 0;
+        __syncthreads();
+        if (b < B) {
+            const int32_t* par = parent + (size_t)b * T;
+            int code = 0;
+            if (r < T) {
+                const int p = par[r];
+                if (r == 0 ? (p != -1) : (p < 0 || p >= r)) code = CONFU_ST_BAD_PARENT;
+            } else if (r < R) {
+                const int o = con_owner[(size_t)b * C + (r - T)];
+                if (o < 0 || o >= T) code = CONFU_ST_BAD_OWNER;
+            }
+            if (code) atomicMax(&s_bad[grp], code == CONFU_ST_BAD_PARENT ? 2 : 1);
+        }
+        __syncthreads();
+        if (b < B) {
+            const int bad = s_bad[grp];
+            const int32_t* par = parent + (size_t)b * T;
+            uint64_t m = 0;
+            if (r < T) {
+                m = 1ull << r;
+                if (!bad) {
+                    int a = par[r];
+                    for (int it = 0; it < T && a >= 0; ++it) { m |= 1ull << a; a = par[a]; }
+                }
+                s_mask[grp][r] = m;
+            }
+            __syncwarp();
+        }
+        __syncthreads();
+        if (b < B) {
+            const int bad = s_bad[grp];
+            uint64_t m = 0;
+            if (r < T) m = s_mask[grp][r];
+            else if (r < R) {
+                m = 1ull << r;
+                if (!bad) m |= s_mask[grp][con_owner[(size_t)b * C + (r - T)]];
+            }
+            pv.mask[(size_t)b * kMaxRows + r] = m;
+            if (r == 0) {
+                const int code = bad == 2 ? CONFU_ST_BAD_PARENT : (bad == 1 ? CONFU_ST_BAD_OWNER : 0);
+                pv.bad[b] = code;
+                if (code && status) status[b] = code;
+                const int64_t keys = (int64_t)prefix_len[b] + R;
+                pv.tiles[b] = code ? 0 : (int32_t)((keys + kTileKeys - 1) / kTileKeys) + (d.S > 0 ? 1 : 0);
+            }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int64_t acc = 0;
+        for (int b = 0; b < B; ++b) {
+            pv.tile_base[b] = acc;
+            acc += (int64_t)pv.tiles[b] * d.Hkv;
+        }
+        pv.tile_base[B] = acc;
+        PlanHeader h;
+        h.B = B; h.Hkv = d.Hkv; h.T = T; h.C = C; h.S = d.S; h.R = R;
+        h.n_tiles = acc;
+        h.n_ctas = (int)(acc < (int64_t)sm_count ? acc : (int64_t)sm_count);
+        h.pad = 0;
+        *pv.hdr = h;
+    }
+    (void)seq_start;
+}
+
+cudaError_t launch_plan(const Ctx* ctx, const confu_dims& d, const int64_t* seq_start, const int32_t* prefix_len,
+                        const int32_t* parent, const int32_t* con_owner, void* plan, int32_t* status,
+                        cudaStream_t st)
+{
+    plan_kernel<<<1, 256, 0, st>>>(d, ctx->sm_count, seq_start, prefix_len, parent, con_owner, plan, status);
+    return cudaGetLastError();
+}
+
+}  // namespace confu

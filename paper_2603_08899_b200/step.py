@@ -1,0 +1,81 @@
+"""One verification step = L x confu_tree_attention + confu_tree_accept + confu_kv_compact, enqueued
+on one stream through the C-ABI binding.  This module only owns buffers and call order; all
+arithmetic runs in the CUDA library."""
+import torch
+
+from . import binding as cb
+
+
+class VerifyStep:
+    def __init__(self, cfg, n_slots, device="cuda", ctx=None):
+        self.cfg = cfg
+        self.n_slots = n_slots
+        self.dev = device
+        self.own_ctx = ctx is None
+        self.ctx = cb.confu_create(torch.device(device).index or 0) if ctx is None else ctx
+        self.dims = cb.make_dims(cfg.B, cfg.Hq, cfg.Hkv, cfg.D, cfg.T, cfg.C, cfg.S, cfg.kv_dtype)
+        B, T = cfg.B, cfg.T
+        u8 = dict(dtype=torch.uint8, device=device)
+        i32 = dict(dtype=torch.int32, device=device)
+        self.ws = torch.empty(cb.confu_workspace_bytes(self.ctx, self.dims), **u8)
+        cb.confu_set_workspace(self.ctx, self.ws)
+        self.plan = torch.empty(cb.confu_plan_bytes(self.ctx, self.dims), **u8)
+        self.accept_ws = torch.empty(cb.confu_accept_workspace_bytes(B, T, cfg.V), **u8)
+        self.status = torch.zeros(B, **i32)
+        self.accept_len = torch.zeros(B, **i32)
+        self.path = torch.zeros(B, cb.MAX_DEPTH + 1, **i32)
+        self.next_token = torch.zeros(B, **i32)
+        self.future_row = torch.zeros(B, **i32)
+        self.counters = torch.zeros(B, 4, **i32)
+        self.new_prefix_len = torch.zeros(B, **i32)
+
+    def close(self):
+        if self.own_ctx:
+            cb.confu_destroy(self.ctx)
+            self.own_ctx = False
+
+    def bind(self, q_layers, k_layers, v_layers, k_soft, v_soft, out_layers, seq_start, prefix_len, parent,
+             con_owner, target_logits, draft_logits, tokens, uniforms):
+        """Remember the (device) tensors of a step; lists have one entry per layer."""
+        self.q, self.k, self.v, self.ks, self.vs, self.out = q_layers, k_layers, v_layers, k_soft, v_soft, out_layers
+        self.seq_start, self.prefix_len, self.parent, self.con_owner = seq_start, prefix_len, parent, con_owner
+        self.tl, self.dl, self.tokens, self.uniforms = target_logits, draft_logits, tokens, uniforms
+        self.k_ptrs = torch.tensor([t.data_ptr() for t in k_layers], dtype=torch.int64, device=self.dev)
+        self.v_ptrs = torch.tensor([t.data_ptr() for t in v_layers], dtype=torch.int64, device=self.dev)
+
+    def run_attention(self, lse_layers=None):
+        cfg = self.cfg
+        cb.confu_tree_plan(self.ctx, self.dims, self.seq_start, self.prefix_len, self.parent, self.con_owner,
+                           self.plan, self.status)
+        for l in range(len(self.q)):
+            cb.confu_tree_attention(self.ctx, self.dims, self.q[l], self.k[l], self.v[l], self.n_slots,
+                                    self.seq_start, self.prefix_len,
+                                    self.ks[l] if self.ks is not None else None,
+                                    self.vs[l] if self.vs is not None else None,
+                                    None, None, self.plan, self.out[l],
+                                    None if lse_layers is None else lse_layers[l], self.status)
+
+    def run_accept(self, temperature, sibling_mode=1):
+        cfg = self.cfg
+        cb.confu_tree_accept(self.ctx, cfg.B, cfg.T, cfg.C, cfg.V, cfg.logit_dtype, self.tl,
+                             self.dl if temperature > 0 else None, self.tokens, self.parent, self.con_owner,
+                             self.uniforms if temperature > 0 else None, temperature, sibling_mode, self.accept_len,
+                             self.path, self.next_token, self.future_row, self.counters, self.accept_ws, self.status)
+
+    def run_compact(self):
+        cb.confu_kv_compact(self.ctx, self.dims, len(self.k), self.k_ptrs, self.v_ptrs, self.seq_start,
+                            self.prefix_len, self.accept_len, self.path, self.new_prefix_len, self.status)
+
+    def run(self, temperature=1.0, sibling_mode=1):
+        """The whole step on the current stream (no host synchronisation)."""
+        self.run_attention()
+        self.run_accept(temperature, sibling_mode)
+        self.run_compact()
+
+    def launches_per_step(self):
+        """Kernels of this library launched by run(): plan + per layer attention + row statistics +
+        walk + compaction."""
+        return 1 + ATTENTION_KERNELS_PER_LAYER * len(self.q) + 3
+
+
+ATTENTION_KERNELS_PER_LAYER = 1
