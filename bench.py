@@ -364,7 +364,7 @@ def run_ours(args, cfg):
     attn_launch_s = ms_attn * 1e-3 / cfg.L
     achieved = a_bytes / attn_launch_s / 1e9
     sbytes = step_bytes(cfg, plen, alen)
-    kname = "attention_tc" if step_mod.ATTENTION_KERNELS_PER_LAYER > 1 else "attention_generic"
+    kname = "attention_tc_kernel" if step_mod.uses_tensor_core_path(cfg) else "attention_generic_kernel"
     cpu = oracle_sample(oracle_prepare(cfg)) if not args.no_cpu_baseline else None
     line = {
         "metric": METRIC, "value": world * args.steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,

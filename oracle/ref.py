@@ -151,7 +151,7 @@ def kv_compact(k_layers, v_layers, seq_start, prefix_len, accept_len, path):
     """In-place compaction of lists of per-layer CPU pools [n_slots, Hkv, D].  Returns new_prefix_len [B]."""
     L = len(k_layers)
     B = prefix_len.shape[0]
-    row_bytes = k_layers[0][0].numel() * k_layers[0].element_size()
+    row_bytes = k_layers[0][0].numel() * k_layers[0].element_size() if L else 1
     for t in list(k_layers) + list(v_layers):
         assert t.device.type == "cpu" and t.is_contiguous()
     kp = (C.c_void_p * L)(*[t.data_ptr() for t in k_layers])

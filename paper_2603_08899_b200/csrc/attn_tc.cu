@@ -1,15 +1,697 @@
-// Tensor-core (tcgen05 + TMA) tree attention -- placeholder until the kernel lands.
+// Tensor-core tree attention for sm_100a: TMA-staged bf16 K/V tiles, tcgen05.mma with TMEM
+// accumulators, warp-specialised online softmax, stream-K split over the ragged batch.
+//
+// One persistent CTA per SM walks a contiguous range of the flat list of 128-key tiles of all
+// (sequence, kv head) pairs.  For a pair the query block is the R rows x G heads that share the kv
+// head: two M tiles of 128 rows (32 rows x G heads each, padded when G < 4).  Per key tile:
+//     S_t = Q_t K^T           tcgen05.mma, A and B from shared memory (K-major, 128B swizzle)
+//     P_t = exp2(S_t*c - m)   one thread per row: tcgen05.ld, mask (last tiles only), tcgen05.st as bf16
+//     O_t += P_t V            tcgen05.mma, A from TMEM, B = V tile in shared memory (MN-major)
+// The two M tiles ping-pong: while the softmax warps of one tile work, the tensor pipe runs the
+// other tile's MMAs.  Prefix tiles need no mask; the ancestor bitmask (one 64-bit word per row,
+// in a register) is applied only to the tiles that hold the tree slots, the ragged tail and the
+// soft-prompt entries.  A range that does not cover a whole pair writes an unnormalised partial
+// (O, m, l) that combine_kernel merges in a fixed order.
+//
+// Every wait on an mbarrier is bounded (wall-clock limit); on expiry the CTA raises an abort flag,
+// every role leaves its loop, tensor memory is released and CONFU_ST_TIMEOUT is reported.
+#include <cuda.h>
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace confu {
 
-bool tc_attention_supported(const confu_dims&) { return false; }
+namespace tc {
 
-cudaError_t launch_attention_tc(const Ctx*, const confu_dims&, const void*, const void*, const void*, int64_t,
-                                const int64_t*, const int32_t*, const void*, const void*, const void*, void*, void*,
-                                float*, int32_t*, cudaStream_t)
+constexpr int kThreads = 384;            // warps 0-3: softmax tile 0, 4-7: softmax tile 1, 8: TMA, 9: MMA
+constexpr int kStages = 4;               // ring of 32 KB slots shared by K and V tiles
+constexpr int kD = 128;
+constexpr int kTileBytes = kTileKeys * kD * 2;      // 32 KB
+constexpr int kHalfTile = kTileBytes / 2;           // one 64-wide half of the head dim: [128 rows][128 B]
+constexpr int kQBytes = 2 * kTileBytes;             // two M tiles
+constexpr uint32_t kTmemCols = 512;                 // S0 | S1 | O0 | O1, 128 columns each; P_t overlays S_t
+constexpr float kRescaleThreshold = 8.f;            // lazy rescale: move the reference max only past 2^8
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct SharedStorage {
+    alignas(1024) uint8_t q[kQBytes];
+    alignas(1024) uint8_t kv[kStages][kTileBytes];
+    alignas(8) uint64_t q_full, q_empty;
+    uint64_t kv_full[kStages], kv_empty[kStages];
+    uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+struct Params {
+    confu_dims d;
+    const int64_t* seq_start;
+    const int32_t* prefix_len;
+    const void* plan;
+    float* partials;
+    __nv_bfloat16* out;
+    float* lse;
+    int32_t* status;
+    int n_mt;            // M tiles in use (R > 32 ? 2 : 1)
+    int G;
+    float c;             // sm_scale * log2(e)
+};
+
+// ------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
 {
-    return cudaErrorNotSupported;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false when the wait expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0) {
+            if (*abort) return false;
+            if (global_ns() - t0 > kWaitLimitNs) { *abort = 1; return false; }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint64_t* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+          "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+          "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
+        : "memory");
+}
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout code 2), descriptor version 1.
+// lbo / sbo in bytes: leading / stride byte offsets of the canonical layout.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; B K-major (QK^T) or MN-major (PV).
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
+
+// ------------------------------------------------------------------------------------ work list
+struct Segment {
+    int b, g;
+    int t0, t1;        // tiles [t0, t1) of this pair
+    int nt, nkt;       // tiles of the pair; key tiles (the soft-prompt tile, if any, is tile nkt)
+    int64_t P;         // prefix length
+    int64_t slot0;     // seq_start
+    int part_slot;     // -1: the range covers the whole pair, write the output directly
+};
+
+struct Walker {
+    const PlanView pv;
+    int64_t f, f1;
+    int cta;
+    const Params& prm;
+    __device__ Walker(const PlanView& v, const Params& p, int cta_) : pv(v), cta(cta_), prm(p)
+    {
+        const int64_t N = v.hdr->n_tiles;
+        const int64_t n = v.hdr->n_ctas;
+        f = (int64_t)cta_ * N / n;
+        f1 = (int64_t)(cta_ + 1) * N / n;
+    }
+    __device__ bool next(Segment& s)
+    {
+        if (f >= f1) return false;
+        int lo = 0, hi = prm.d.B;                  // largest b with tile_base[b] <= f
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (pv.tile_base[mid] <= f) lo = mid; else hi = mid;
+        }
+        s.b = lo;
+        s.nt = pv.tiles[lo];
+        const int64_t local = f - pv.tile_base[lo];
+        s.g = (int)(local / s.nt);
+        s.t0 = (int)(local % s.nt);
+        const int64_t room = f1 - f;
+        s.t1 = (int)((int64_t)(s.nt - s.t0) <= room ? s.nt : s.t0 + room);
+        s.nkt = s.nt - (prm.d.S > 0 ? 1 : 0);
+        s.P = prm.prefix_len[lo];
+        s.slot0 = prm.seq_start[lo];
+        const bool whole = s.t0 == 0 && s.t1 == s.nt;
+        s.part_slot = whole ? -1 : 2 * cta + (s.t1 < s.nt ? 1 : 0);
+        f += s.t1 - s.t0;
+        return true;
+    }
+};
+
+// ------------------------------------------------------------------------------------ roles
+__device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanView& pv, const CUtensorMap* q_map,
+                              const CUtensorMap* k_map, const CUtensorMap* v_map, const CUtensorMap* ks_map,
+                              const CUtensorMap* vs_map)
+{
+    Walker w(pv, prm, blockIdx.x);
+    Segment s;
+    uint32_t ring = 0;                 // running count of ring slots filled
+    uint32_t seg = 0;
+    const int R = prm.d.T + prm.d.C;
+    const uint32_t q_box_bytes = 32u * prm.G * 128u;
+    while (w.next(s)) {
+        // Q of this pair (both M tiles, two 64-wide halves each)
+        if (!mbar_wait(&sh.q_empty, (seg & 1) ^ 1, &sh.abort)) return;
+        mbar_arrive_expect_tx(&sh.q_full, 2u * prm.n_mt * q_box_bytes);
+        for (int t = 0; t < prm.n_mt; ++t)
+            for (int kb = 0; kb < 2; ++kb)
+                tma_load_3d(sh.q + (t * 2 + kb) * kHalfTile, q_map, &sh.q_full, kb * 64, s.g * prm.G, s.b * R + 32 * t);
+        for (int t = s.t0; t < s.t1; ++t) {
+            const bool soft = t >= s.nkt;
+            const int z = soft ? 0 : (int)(s.slot0 + (int64_t)t * kTileKeys);
+            for (int which = 0; which < 2; ++which) {       // K then V
+                const uint32_t st = ring % kStages;
+                if (!mbar_wait(&sh.kv_empty[st], ((ring / kStages) & 1) ^ 1, &sh.abort)) return;
+                mbar_arrive_expect_tx(&sh.kv_full[st], kTileBytes);
+                const CUtensorMap* m = which == 0 ? (soft ? ks_map : k_map) : (soft ? vs_map : v_map);
+                tma_load_3d(sh.kv[st], m, &sh.kv_full[st], 0, s.g, z);
+                tma_load_3d(sh.kv[st] + kHalfTile, m, &sh.kv_full[st], 64, s.g, z);
+                ++ring;
+            }
+        }
+        ++seg;
+    }
+}
+
+__device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem)
+{
+    Walker w(pv, prm, blockIdx.x);
+    Segment s;
+    uint32_t ring = 0, seg = 0;
+    uint32_t n_s[2] = {0, 0};          // S tiles produced per M tile (phase of s_full)
+    uint32_t n_p[2] = {0, 0};          // P tiles consumed per M tile (phase of p_full)
+    const uint32_t q_addr = smem_u32(sh.q);
+
+    auto issue_qk = [&](int t, uint32_t k_addr) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t off = (uint32_t)(i >> 2) * kHalfTile + (uint32_t)(i & 3) * 32u;
+            mma_ss(tmem + t * 128, smem_desc(q_addr + t * kTileBytes + off, 16, 1024),
+                   smem_desc(k_addr + off, 16, 1024), kIdescQK, i > 0 ? 1u : 0u);
+        }
+        tc_commit(&sh.s_full[t]);
+        ++n_s[t];
+    };
+    auto issue_pv = [&](int t, uint32_t v_addr, bool first_of_segment) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            mma_ts(tmem + 256 + t * 128, tmem + t * 128 + i * 8, smem_desc(v_addr + i * 2048u, kHalfTile, 1024), kIdescPV,
+                   (first_of_segment && i == 0) ? 0u : 1u);
+    };
+
+    while (w.next(s)) {
+        const int n_tiles = s.t1 - s.t0;
+        if (!mbar_wait(&sh.q_full, seg & 1, &sh.abort)) return;
+        // accumulators of the previous pair must have been read out
+        for (int t = 0; t < prm.n_mt; ++t)
+            if (!mbar_wait(&sh.o_free[t], (seg & 1) ^ 1, &sh.abort)) return;
+        tc_fence_after();
+        // first key tile: S_0, S_1
+        uint32_t k_slot = ring % kStages;
+        if (!mbar_wait(&sh.kv_full[k_slot], (ring / kStages) & 1, &sh.abort)) return;
+        tc_fence_after();
+        for (int t = 0; t < prm.n_mt; ++t) issue_qk(t, smem_u32(sh.kv[k_slot]));
+        tc_commit(&sh.kv_empty[k_slot]);
+        ++ring;
+        if (n_tiles == 1) tc_commit(&sh.q_empty);
+        for (int j = 0; j < n_tiles; ++j) {
+            const uint32_t v_slot = ring % kStages;
+            if (!mbar_wait(&sh.kv_full[v_slot], (ring / kStages) & 1, &sh.abort)) return;
+            ++ring;
+            const bool more = j + 1 < n_tiles;
+            uint32_t nk_slot = 0;
+            if (more) {
+                nk_slot = ring % kStages;
+                if (!mbar_wait(&sh.kv_full[nk_slot], (ring / kStages) & 1, &sh.abort)) return;
+                ++ring;
+            }
+            for (int t = 0; t < prm.n_mt; ++t) {
+                if (!mbar_wait(&sh.p_full[t], n_p[t] & 1, &sh.abort)) return;
+                ++n_p[t];
+                tc_fence_after();
+                issue_pv(t, smem_u32(sh.kv[v_slot]), j == 0);
+                if (!more) tc_commit(&sh.o_done[t]);
+                if (more) issue_qk(t, smem_u32(sh.kv[nk_slot]));
+            }
+            tc_commit(&sh.kv_empty[v_slot]);
+            if (more) {
+                tc_commit(&sh.kv_empty[nk_slot]);
+                if (j + 2 == n_tiles) tc_commit(&sh.q_empty);       // last QK of the pair has been issued
+            }
+        }
+        ++seg;
+    }
+}
+
+// Which of the 128 keys of tile `t` may row r see.  lo: keys 0..63 of the tile, hi: 64..127.
+__device__ __forceinline__ void visible_bits(const Segment& s, int t, int R, int T, int S, int r, bool row_valid,
+                                             uint64_t mask, uint64_t& lo, uint64_t& hi)
+{
+    if (!row_valid) { lo = hi = ~0ull; return; }
+    if (t >= s.nkt) {                          // soft-prompt tile: contemplate rows only, S entries
+        const bool sees = r >= T;
+        lo = sees ? (S >= 64 ? ~0ull : ((1ull << S) - 1)) : 0ull;
+        hi = sees ? (S > 64 ? (S >= 128 ? ~0ull : ((1ull << (S - 64)) - 1)) : 0ull) : 0ull;
+        return;
+    }
+    const int64_t off = s.P - (int64_t)t * kTileKeys;      // position of tree slot 0 inside this tile (may be < 0 or >= 128)
+    // prefix part: keys [0, off)
+    unsigned __int128 v = 0;
+    if (off >= 128) v = ~(unsigned __int128)0;
+    else if (off > 0) v = (((unsigned __int128)1) << off) - 1;
+    // tree part: bit j of mask at position off + j
+    const unsigned __int128 m = (unsigned __int128)(R >= 64 ? mask : (mask & ((1ull << R) - 1)));
+    if (off >= 0) { if (off < 128) v |= m << off; }
+    else if (off > -64) v |= m >> (-off);
+    lo = (uint64_t)v;
+    hi = (uint64_t)(v >> 64);
+}
+
+__device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem, int t /*M tile*/)
+{
+    const int lane_row = threadIdx.x & 127;                 // row of the M tile = TMEM lane
+    const int warp_in_wg = (threadIdx.x >> 5) & 3;
+    const uint32_t lane_base = (uint32_t)(warp_in_wg * 32) << 16;
+    const uint32_t s_addr = tmem + lane_base + t * 128;
+    const uint32_t o_addr = tmem + lane_base + 256 + t * 128;
+    const int G = prm.G, T = prm.d.T, R = prm.d.T + prm.d.C, S = prm.d.S, Hq = prm.d.Hq;
+    const int r = 32 * t + lane_row / G, hl = lane_row % G;
+    const bool row_valid = lane_row < 32 * G && r < R;
+    const float c = prm.c;
+
+    Walker w(pv, prm, blockIdx.x);
+    Segment s;
+    uint32_t n_s = 0, seg = 0;
+    while (w.next(s)) {
+        const uint64_t mask = row_valid ? pv.mask[(size_t)s.b * kMaxRows + r] : 0ull;
+        float m_ref = -INFINITY, l = 0.f;
+        for (int tile = s.t0; tile < s.t1; ++tile) {
+            if (!mbar_wait(&sh.s_full[t], n_s & 1, &sh.abort)) return;
+            ++n_s;
+            tc_fence_after();
+            uint32_t sv[128];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(s_addr + q4 * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[q4 * 32]));
+            tc_wait_ld();
+            const bool masked = tile >= s.nkt || (int64_t)(tile + 1) * kTileKeys > s.P;
+            if (masked) {
+                uint64_t lo, hi;
+                visible_bits(s, tile, R, T, S, r, row_valid, mask, lo, hi);
+#pragma unroll
+                for (int j = 0; j < 64; ++j) {
+                    if (!((lo >> j) & 1ull)) sv[j] = 0xff800000u;            // -inf
+                    if (!((hi >> j) & 1ull)) sv[64 + j] = 0xff800000u;
+                }
+            }
+            float mx = __uint_as_float(sv[0]);
+#pragma unroll
+            for (int j = 1; j < 128; ++j) mx = fmaxf(mx, __uint_as_float(sv[j]));
+            const float m_new = fmaxf(m_ref, mx * c);
+            if (tile == s.t0) {
+                m_ref = m_new;
+            } else {
+                const bool move = m_new - m_ref > kRescaleThreshold;         // false when both are -inf (NaN)
+                if (__any_sync(0xffffffffu, move)) {
+                    const float alpha = move ? ex2(m_ref - m_new) : 1.f;
+                    if (move) { m_ref = m_new; l *= alpha; }
+                    // S_full of this tile implies the previous PV of this M tile has completed
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t ov[32];
+                        tmem_ld32(o_addr + q4 * 32, ov);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
+                        tmem_st32(o_addr + q4 * 32, ov);
+                    }
+                }
+            }
+            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            float sum = 0.f;
+            uint32_t pk[64];
+#pragma unroll
+            for (int j = 0; j < 64; ++j) {
+                const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), c, neg_m));
+                const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), c, neg_m));
+                sum += p0 + p1;
+                pk[j] = pack_bf16(p0, p1);
+            }
+            l += sum;
+            tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+            tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sh.p_full[t]);
+        }
+        // ---- epilogue of this pair / range ----
+        if (!mbar_wait(&sh.o_done[t], seg & 1, &sh.abort)) return;
+        tc_fence_after();
+        const int h = s.g * G + hl;
+        if (s.part_slot < 0) {
+            const float inv_l = 1.f / l;
+            __nv_bfloat16* orow = prm.out + (((size_t)s.b * R + r) * Hq + h) * kD;
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                uint32_t ov[32];
+                tmem_ld32(o_addr + q4 * 32, ov);
+                tc_wait_ld();
+                if (row_valid) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 pkt;
+                        pkt.x = pack_bf16(__uint_as_float(ov[8 * j + 0]) * inv_l, __uint_as_float(ov[8 * j + 1]) * inv_l);
+                        pkt.y = pack_bf16(__uint_as_float(ov[8 * j + 2]) * inv_l, __uint_as_float(ov[8 * j + 3]) * inv_l);
+                        pkt.z = pack_bf16(__uint_as_float(ov[8 * j + 4]) * inv_l, __uint_as_float(ov[8 * j + 5]) * inv_l);
+                        pkt.w = pack_bf16(__uint_as_float(ov[8 * j + 6]) * inv_l, __uint_as_float(ov[8 * j + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(orow + q4 * 32 + j * 8) = pkt;
+                    }
+                }
+            }
+            if (row_valid && prm.lse)
+                prm.lse[((size_t)s.b * R + r) * Hq + h] = (m_ref + log2f(l)) * 0.6931471805599453f;
+        } else {
+            float* slot = prm.partials + (size_t)s.part_slot * (partial_slot_bytes() / sizeof(float));
+            float* prow = slot + (size_t)(t * 128 + lane_row) * kPartD;
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                uint32_t ov[32];
+                tmem_ld32(o_addr + q4 * 32, ov);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    *reinterpret_cast<uint4*>(prow + q4 * 32 + j * 4) = make_uint4(ov[4 * j], ov[4 * j + 1], ov[4 * j + 2], ov[4 * j + 3]);
+            }
+            float* ml = slot + (size_t)kPartRows * kPartD;
+            ml[t * 128 + lane_row] = m_ref;
+            ml[kPartRows + t * 128 + lane_row] = l;
+        }
+        tc_fence_before();
+        mbar_arrive(&sh.o_free[t]);
+        ++seg;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                    const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap ks_map,
+                    const __grid_constant__ CUtensorMap vs_map, const Params prm)
+{
+    extern __shared__ uint8_t smem_raw[];
+    SharedStorage& sh = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
+    if ((int)blockIdx.x >= pv.hdr->n_ctas) return;
+    const int warp = threadIdx.x >> 5;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sh.q_full, 1);
+        mbar_init(&sh.q_empty, 1);
+        for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&sh.s_full[t], 1);
+            mbar_init(&sh.p_full[t], 128);
+            mbar_init(&sh.o_done[t], 1);
+            mbar_init(&sh.o_free[t], 128);
+        }
+        sh.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 9) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh.tmem_base;
+
+    if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        const int t = warp >> 2;
+        if (t < prm.n_mt) softmax_role(sh, prm, pv, tmem, t);
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        if (warp == 8) {
+            if ((threadIdx.x & 31) == 0) producer_role(sh, prm, pv, &q_map, &k_map, &v_map, &ks_map, &vs_map);
+        } else if (warp == 9) {
+            if ((threadIdx.x & 31) == 0) mma_role(sh, prm, pv, tmem);
+        }
+        __syncwarp();
+    }
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (sh.abort) {
+        // give copies that may still be in flight time to land before the CTA's shared memory goes away
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        if (threadIdx.x == 0 && prm.status)
+            for (int b = 0; b < prm.d.B; ++b) prm.status[b] = CONFU_ST_TIMEOUT;
+        __syncthreads();
+    }
+    if (warp == 9) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// Merge of the split-KV partials of one (sequence, kv head) pair, in CTA order (deterministic).
+__global__ void __launch_bounds__(128) combine_kernel(const Params prm)
+{
+    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
+    const int pair = blockIdx.x, t = blockIdx.y;
+    const int b = pair / prm.d.Hkv, g = pair % prm.d.Hkv;
+    const int nt = pv.tiles[b];
+    if (nt == 0 || t >= prm.n_mt) return;
+    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
+    const int64_t F = pv.tile_base[b] + (int64_t)g * nt;
+    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
+    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
+    const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
+    const int lane_row = threadIdx.x;
+    const int r = 32 * t + lane_row / G, hl = lane_row % G;
+    if (!(lane_row < 32 * G && r < R)) return;
+    const size_t slot_floats = partial_slot_bytes() / sizeof(float);
+    const int row = t * 128 + lane_row;
+    float M = -INFINITY;
+    for (int cta = c_first; cta <= c_last; ++cta) {
+        const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
+        M = fmaxf(M, slot[(size_t)kPartRows * kPartD + row]);
+    }
+    float acc[kPartD];
+#pragma unroll
+    for (int j = 0; j < kPartD; ++j) acc[j] = 0.f;
+    float L = 0.f;
+    for (int cta = c_first; cta <= c_last; ++cta) {
+        const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
+        const float m = slot[(size_t)kPartRows * kPartD + row];
+        const float w = (m == -INFINITY) ? 0.f : ex2(m - M);
+        L += w * slot[(size_t)kPartRows * kPartD + kPartRows + row];
+        const float4* prow = reinterpret_cast<const float4*>(slot + (size_t)row * kPartD);
+#pragma unroll
+        for (int j = 0; j < kPartD / 4; ++j) {
+            const float4 v = prow[j];
+            acc[4 * j] += w * v.x; acc[4 * j + 1] += w * v.y; acc[4 * j + 2] += w * v.z; acc[4 * j + 3] += w * v.w;
+        }
+    }
+    const float inv_l = 1.f / L;
+    const int h = g * G + hl;
+    __nv_bfloat16* orow = prm.out + (((size_t)b * R + r) * Hq + h) * kD;
+#pragma unroll
+    for (int j = 0; j < kPartD / 8; ++j) {
+        uint4 pkt;
+        pkt.x = pack_bf16(acc[8 * j] * inv_l, acc[8 * j + 1] * inv_l);
+        pkt.y = pack_bf16(acc[8 * j + 2] * inv_l, acc[8 * j + 3] * inv_l);
+        pkt.z = pack_bf16(acc[8 * j + 4] * inv_l, acc[8 * j + 5] * inv_l);
+        pkt.w = pack_bf16(acc[8 * j + 6] * inv_l, acc[8 * j + 7] * inv_l);
+        *reinterpret_cast<uint4*>(orow + j * 8) = pkt;
+    }
+    if (prm.lse) prm.lse[((size_t)b * R + r) * Hq + h] = (M + log2f(L)) * 0.6931471805599453f;
+}
+
+// ------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// [rows][heads][128] bf16 tensor, box = box_rows x box_heads x 64 elements, 128-byte swizzle
+static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t heads, uint32_t box_rows,
+                     uint32_t box_heads)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)kD, heads, rows};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, heads * kD * 2};
+    const cuuint32_t box[3] = {64, box_heads, box_rows};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace tc
+
+bool tc_attention_supported(const confu_dims& d)
+{
+    static const bool force_generic = getenv("CONFU_FORCE_GENERIC") != nullptr;     // debugging aid
+    if (force_generic) return false;
+    const int G = d.Hq / d.Hkv;
+    return d.kv_dtype == CONFU_BF16 && d.D == 128 && G <= 4 && d.S <= 128;
+}
+
+cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
+                                const void* v_cache, int64_t n_slots, const int64_t* seq_start,
+                                const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
+                                void* partials, void* out, float* lse, int32_t* status, cudaStream_t st)
+{
+    using namespace tc;
+    const int R = d.T + d.C, G = d.Hq / d.Hkv;
+    CUtensorMap q_map, k_map, v_map, ks_map, vs_map;
+    bool ok = make_map(&q_map, q, (uint64_t)d.B * R, d.Hq, 32, G) && make_map(&k_map, k_cache, n_slots, d.Hkv, kTileKeys, 1) &&
+              make_map(&v_map, v_cache, n_slots, d.Hkv, kTileKeys, 1);
+    if (d.S > 0) ok = ok && make_map(&ks_map, k_soft, d.S, d.Hkv, kTileKeys, 1) && make_map(&vs_map, v_soft, d.S, d.Hkv, kTileKeys, 1);
+    else { ks_map = k_map; vs_map = v_map; }
+    if (!ok) return cudaErrorInvalidValue;
+    Params prm;
+    prm.d = d;
+    prm.seq_start = seq_start;
+    prm.prefix_len = prefix_len;
+    prm.plan = plan;
+    prm.partials = (float*)partials;
+    prm.out = (__nv_bfloat16*)out;
+    prm.lse = lse;
+    prm.status = status;
+    prm.n_mt = R > 32 ? 2 : 1;
+    prm.G = G;
+    prm.c = (d.sm_scale != 0.f ? d.sm_scale : 1.f / sqrtf((float)d.D)) * 1.4426950408889634f;
+    const size_t smem = sizeof(SharedStorage) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    attention_tc_kernel<<<ctx->sm_count, kThreads, smem, st>>>(q_map, k_map, v_map, ks_map, vs_map, prm);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    combine_kernel<<<dim3(d.B * d.Hkv, prm.n_mt), 128, 0, st>>>(prm);
+    return cudaGetLastError();
 }
 
 }  // namespace confu

@@ -75,7 +75,16 @@ class VerifyStep:
     def launches_per_step(self):
         """Kernels of this library launched by run(): plan + per layer attention + row statistics +
         walk + compaction."""
-        return 1 + ATTENTION_KERNELS_PER_LAYER * len(self.q) + 3
+        return 1 + attention_kernels_per_layer(self.cfg) * len(self.q) + 3
 
 
-ATTENTION_KERNELS_PER_LAYER = 1
+def uses_tensor_core_path(cfg):
+    """Mirror of the library's dispatch rule: bf16, head dim 128, at most 4 query heads per KV head."""
+    import os
+    return (cfg.kv_dtype == torch.bfloat16 and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
+            and "CONFU_FORCE_GENERIC" not in os.environ)
+
+
+def attention_kernels_per_layer(cfg):
+    """Tensor-core path: attention + split combine; generic path: one kernel."""
+    return 2 if uses_tensor_core_path(cfg) else 1
