@@ -118,12 +118,13 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- CPU oracle leg
-def oracle_prepare(cfg, target_visits=100e6):
+def oracle_prepare(cfg, target_visits=1e9, max_seqs=32):
     """Inputs of the bounded oracle sample (generation is not timed).  The number of sampled attention
-    rows is set so that the sample visits about `target_visits` (row, key) pairs: ~10 s on 8 cores."""
+    rows is set so that the sample visits at most about `target_visits` (row, key) pairs (capped at
+    every output row of one layer of the sampled sequences): 10-20 s of work on 16 cores by default."""
     parent, owner = inputs.trees(cfg)
     plen = inputs.prefix_lens(cfg)
-    nseq = min(cfg.B, 4)
+    nseq = min(cfg.B, max_seqs)
     sub = inputs.scaled(cfg, B=nseq)
     sp = {"cfg": cfg, "nseq": nseq, "plen_all": plen, "parent": parent[:nseq].contiguous(),
           "owner": owner[:nseq].contiguous(), "plen": plen[:nseq].contiguous()}
@@ -141,7 +142,7 @@ def oracle_prepare(cfg, target_visits=100e6):
 
 def oracle_sample(sp):
     """Times the fp64 oracle, as it stands, on a bounded sample of the workload and scales the result
-    to one whole step.  Sample: a few hundred (row, head) outputs of layer 0 for up to 4 sequences
+    to one whole step.  Sample: (row, head) outputs of layer 0 of the sampled sequences
     (attention cost is proportional to the visible keys, which the scaling uses), the acceptance walk
     of those sequences at full vocabulary, and the compaction of one layer."""
     from oracle import ref
@@ -170,7 +171,7 @@ def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sp = oracle_prepare(cfg, target_visits=25e6)
+    sp = oracle_prepare(cfg, target_visits=25e6, max_seqs=4)
     for i in range(args.warmup):
         oracle_sample(sp)
     t0 = time.perf_counter()
@@ -292,67 +293,72 @@ def run_ours(args, cfg):
     ms_plan, ms_attn, ms_acc, ms_cmp = part(0, 1), part(1, 2), part(2, 3), part(3, 4)
     alen = step.accept_len.float().mean().item()
 
-    # ---- end to end: this step's inputs come from pinned host memory, results go back ----
-    h = {"q": [t.cpu().pin_memory() for t in step.q],
-         "krows": [], "vrows": [],
-         "tl": step.tl.cpu().pin_memory(), "dl": step.dl.cpu().pin_memory(),
-         "tok": host["tok"].pin_memory(), "u": host["u"].pin_memory(), "parent": host["parent"].pin_memory(),
-         "owner": host["owner"].pin_memory()}
-    R = cfg.R
-    idx = torch.cat([torch.arange(int(host["seq_start"][b]) + int(plen[b]), int(host["seq_start"][b]) + int(plen[b]) + R)
-                     for b in range(cfg.B)]).to(device)
-    for l in range(cfg.L):
-        h["krows"].append(step.k[l][idx].view(cfg.B, R, cfg.Hkv, cfg.D).cpu().pin_memory())
-        h["vrows"].append(step.v[l][idx].view(cfg.B, R, cfg.Hkv, cfg.D).cpu().pin_memory())
-    d_krows = torch.empty_like(h["krows"][0], device=device)
-    d_vrows = torch.empty_like(h["vrows"][0], device=device)
-    res_host = {k: torch.empty_like(getattr(step, k), device="cpu").pin_memory()
-                for k in ("accept_len", "path", "next_token", "future_row", "new_prefix_len", "status")}
-    h2d = sum(t.numel() * t.element_size() for t in h["q"] + h["krows"] + h["vrows"]) + \
-        sum(h[k].numel() * h[k].element_size() for k in ("tl", "dl", "tok", "u", "parent", "owner"))
-    d2h = sum(t.numel() * t.element_size() for t in res_host.values())
-
-    def e2e_step():
-        step.parent.copy_(h["parent"], non_blocking=True)
-        if cfg.C:
-            step.con_owner.copy_(h["owner"], non_blocking=True)
-        step.tokens.copy_(h["tok"], non_blocking=True)
-        step.uniforms.copy_(h["u"], non_blocking=True)
-        cb.confu_tree_plan(step.ctx, step.dims, step.seq_start, step.prefix_len, step.parent, step.con_owner,
-                           step.plan, step.status)
+    def measure_e2e():
+        # ---- end to end: this step's inputs come from pinned host memory, results go back ----
+        h = {"q": [t.cpu().pin_memory() for t in step.q],
+             "krows": [], "vrows": [],
+             "tl": step.tl.cpu().pin_memory(), "dl": step.dl.cpu().pin_memory(),
+             "tok": host["tok"].pin_memory(), "u": host["u"].pin_memory(), "parent": host["parent"].pin_memory(),
+             "owner": host["owner"].pin_memory()}
+        R = cfg.R
+        idx = torch.cat([torch.arange(int(host["seq_start"][b]) + int(plen[b]), int(host["seq_start"][b]) + int(plen[b]) + R)
+                         for b in range(cfg.B)]).to(device)
         for l in range(cfg.L):
-            step.q[l].copy_(h["q"][l], non_blocking=True)
-            d_krows.copy_(h["krows"][l], non_blocking=True)
-            d_vrows.copy_(h["vrows"][l], non_blocking=True)
-            cb.confu_kv_append(step.ctx, step.dims, d_krows, d_vrows, step.k[l], step.v[l], step.seq_start,
-                               step.prefix_len)
-            cb.confu_tree_attention(step.ctx, step.dims, step.q[l], step.k[l], step.v[l], step.n_slots,
-                                    step.seq_start, step.prefix_len, step.ks[l] if step.ks else None,
-                                    step.vs[l] if step.vs else None, None, None, step.plan, step.out[l], None,
-                                    step.status)
-        step.tl.copy_(h["tl"], non_blocking=True)
-        step.dl.copy_(h["dl"], non_blocking=True)
-        step.run_accept(1.0)
-        step.run_compact()
-        for k, t in res_host.items():
-            t.copy_(getattr(step, k), non_blocking=True)
+            h["krows"].append(step.k[l][idx].view(cfg.B, R, cfg.Hkv, cfg.D).cpu().pin_memory())
+            h["vrows"].append(step.v[l][idx].view(cfg.B, R, cfg.Hkv, cfg.D).cpu().pin_memory())
+        d_krows = torch.empty_like(h["krows"][0], device=device)
+        d_vrows = torch.empty_like(h["vrows"][0], device=device)
+        res_host = {k: torch.empty_like(getattr(step, k), device="cpu").pin_memory()
+                    for k in ("accept_len", "path", "next_token", "future_row", "new_prefix_len", "status")}
+        h2d = sum(t.numel() * t.element_size() for t in h["q"] + h["krows"] + h["vrows"]) + \
+            sum(h[k].numel() * h[k].element_size() for k in ("tl", "dl", "tok", "u", "parent", "owner"))
+        d2h = sum(t.numel() * t.element_size() for t in res_host.values())
 
-    n_e2e = max(2, min(args.steps, 5))
-    e2e_step()
-    torch.cuda.synchronize()
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(n_e2e):
+        def e2e_step():
+            step.parent.copy_(h["parent"], non_blocking=True)
+            if cfg.C:
+                step.con_owner.copy_(h["owner"], non_blocking=True)
+            step.tokens.copy_(h["tok"], non_blocking=True)
+            step.uniforms.copy_(h["u"], non_blocking=True)
+            cb.confu_tree_plan(step.ctx, step.dims, step.seq_start, step.prefix_len, step.parent, step.con_owner,
+                               step.plan, step.status)
+            for l in range(cfg.L):
+                step.q[l].copy_(h["q"][l], non_blocking=True)
+                d_krows.copy_(h["krows"][l], non_blocking=True)
+                d_vrows.copy_(h["vrows"][l], non_blocking=True)
+                cb.confu_kv_append(step.ctx, step.dims, d_krows, d_vrows, step.k[l], step.v[l], step.seq_start,
+                                   step.prefix_len)
+                cb.confu_tree_attention(step.ctx, step.dims, step.q[l], step.k[l], step.v[l], step.n_slots,
+                                        step.seq_start, step.prefix_len, step.ks[l] if step.ks else None,
+                                        step.vs[l] if step.vs else None, None, None, step.plan, step.out[l], None,
+                                        step.status)
+            step.tl.copy_(h["tl"], non_blocking=True)
+            step.dl.copy_(h["dl"], non_blocking=True)
+            step.run_accept(1.0)
+            step.run_compact()
+            for k, t in res_host.items():
+                t.copy_(getattr(step, k), non_blocking=True)
+
+        n_e2e = max(2, min(args.steps, 5))
         e2e_step()
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tt = torch.tensor([e2e_ms], device=device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = tt.item()
-    e2e_value = world * n_e2e / (e2e_ms * 1e-3)
+        torch.cuda.synchronize()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if dist is not None:
+            tt = torch.tensor([e2e_ms], device=device)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_ms = tt.item()
+        e2e_value = world * n_e2e / (e2e_ms * 1e-3)
+
+        return e2e_value, e2e_ms / n_e2e, n_e2e, h2d, d2h
+
+    e2e = None if args.no_e2e else measure_e2e()
 
     if rank != 0:
         if dist is not None:
@@ -386,10 +392,11 @@ def run_ours(args, cfg):
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "tensor_tflops": a_flops / attn_launch_s / 1e12,
                      "tensor_frac_of_bf16_peak": a_flops / attn_launch_s / 1e12 / peaks["bf16_tflops"]},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms / n_e2e, "steps": n_e2e,
-                "note": "per step: Q, the R rows' K/V (all layers), both logit matrices, tree arrays and uniforms "
-                        "copied from pinned host memory; results copied back; the prefix KV cache is resident state"},
+        "e2e": None if e2e is None else {
+            "value": e2e[0], "unit": UNIT, "h2d_bytes_per_step": e2e[3], "d2h_bytes_per_step": e2e[4],
+            "ms_per_step": e2e[1], "steps": e2e[2],
+            "note": "per step: Q, the R rows' K/V (all layers), both logit matrices, tree arrays and uniforms "
+                    "copied from pinned host memory; results copied back; the prefix KV cache is resident state"},
         "gpu_launches": args.steps * step.launches_per_step(),
         "clocks": clocks,
     }
@@ -409,9 +416,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="batch32", choices=list(inputs.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--layers", type=int, default=0, help="cut the layer count (profiling runs; named in config.workload)")
+    ap.add_argument("--batch", type=int, default=0, help="cut the batch (profiling runs; named in config.workload)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = inputs.CONFIGS[args.config]
+    cut = {k: v for k, v in (("L", args.layers), ("B", args.batch)) if v > 0}
+    if cut:
+        cfg = inputs.scaled(cfg, name=cfg.name + "[" + ",".join(f"{k}={v}" for k, v in cut.items()) + "]", **cut)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
