@@ -62,12 +62,50 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
 
 
-def profile_traffic(kernel):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if there is one."""
-    p = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(p):
-        return json.load(open(p)).get(kernel)
-    return None
+KERNEL_SOURCES = {"attention_tc_kernel": "attn_tc.cu", "attention_generic_kernel": "attn_generic.cu"}
+
+
+def kernel_source_hash(kernel):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2603_08899_b200", "csrc", KERNEL_SOURCES[kernel])
+    return hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+
+
+def profile_traffic(kernel, workload):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from the
+    committed ncu summary of this workload; None when there is no summary or when the kernel's source has
+    changed since the counters were taken (the summary records the source's hash)."""
+    p = os.path.join(ROOT, "profiles", f"{kernel}_{workload}_L1.md")
+    if not os.path.exists(p):
+        return None
+    traffic = sha = None
+    for line in open(p):
+        if line.startswith("traffic_bytes_per_launch:"):
+            traffic = int(line.split(":")[1])
+        if line.startswith("kernel_source_sha256_16:"):
+            sha = line.split(":")[1].strip()
+    if traffic is None or sha != kernel_source_hash(kernel):
+        return None
+    return traffic
+
+
+def rank_config(cfg, rank):
+    """Weak scaling by sequence: every rank verifies its own seeded batch of the same shape."""
+    return inputs.scaled(cfg, seed=cfg.seed + 1000 * rank) if rank else cfg
+
+
+def max_over_ranks(ms, dist, device):
+    """Timing of a multi-rank run: the slowest rank's device time (no other collective is on the path)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(world, steps, total_ms):
+    """Whole-job throughput: steps of all ranks over the slowest rank's time."""
+    return world * steps / (total_ms * 1e-3)
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -194,8 +232,7 @@ def run_reference(args, cfg):
 # ----------------------------------------------------------------------------- GPU leg
 def build_workload(cfg, device, rank):
     from paper_2603_08899_b200.step import VerifyStep
-    if rank:
-        cfg = inputs.scaled(cfg, seed=cfg.seed + 1000 * rank)      # every rank its own batch (weak scaling)
+    cfg = rank_config(cfg, rank)
     parent, owner = inputs.trees(cfg)
     plen = inputs.prefix_lens(cfg)
     seq_start, n_slots = inputs.cache_layout(cfg, plen)
@@ -283,11 +320,7 @@ def run_ours(args, cfg):
     t_end.record()
     barrier()
     clocks = sampler.stop() if sampler else None
-    total_ms = t_begin.elapsed_time(t_end)
-    if dist is not None:
-        tt = torch.tensor([total_ms], device=device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = tt.item()
+    total_ms = max_over_ranks(t_begin.elapsed_time(t_end), dist, device)
     ms_step = total_ms / args.steps
     part = lambda a, b: statistics.mean(ev[i][a].elapsed_time(ev[i][b]) for i in range(args.steps))  # noqa: E731
     ms_plan, ms_attn, ms_acc, ms_cmp = part(0, 1), part(1, 2), part(2, 3), part(3, 4)
@@ -349,12 +382,8 @@ def run_ours(args, cfg):
             e2e_step()
         e1.record()
         barrier()
-        e2e_ms = e0.elapsed_time(e1)
-        if dist is not None:
-            tt = torch.tensor([e2e_ms], device=device)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = tt.item()
-        e2e_value = world * n_e2e / (e2e_ms * 1e-3)
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, device)
+        e2e_value = aggregate_value(world, n_e2e, e2e_ms)
 
         return e2e_value, e2e_ms / n_e2e, n_e2e, h2d, d2h
 
@@ -373,7 +402,7 @@ def run_ours(args, cfg):
     kname = "attention_tc_kernel" if step_mod.uses_tensor_core_path(cfg) else "attention_generic_kernel"
     cpu = oracle_sample(oracle_prepare(cfg)) if not args.no_cpu_baseline else None
     line = {
-        "metric": METRIC, "value": world * args.steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": aggregate_value(world, args.steps, total_ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "layers": cfg.L, "heads": f"{cfg.Hq}q/{cfg.Hkv}kv", "head_dim": cfg.D,
@@ -387,7 +416,7 @@ def run_ours(args, cfg):
                    "step_frac_of_hbm_roofline": sbytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                    "mean_accept_len": alen, "status_ok": status_ok, "spot_check_vs_oracle": checked},
         "roofline": {"bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": profile_traffic(kname),
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": profile_traffic(kname, inputs.CONFIGS[args.config].name),
                      "peak_source": peaks["source"], "bytes_per_launch": a_bytes, "launch_ms": attn_launch_s * 1e3,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "tensor_tflops": a_flops / attn_launch_s / 1e12,
