@@ -178,6 +178,29 @@ int confu_tree_accept(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V
                       int32_t* counters, void* workspace, size_t workspace_bytes,
                       int32_t* status, void* stream);
 
+/*
+ * confu_tree_accept without any allocation (the paper has no counterpart: this is a packaging
+ * variant for hosts that cannot call cudaMalloc -- an engine whose pool owns the device, a plugin
+ * that gets streams but no allocator, a loop that must not synchronise).  Same arguments, meaning,
+ * outputs and error codes as confu_tree_accept, minus the context and the workspace: the row
+ * statistics go to a fixed array inside the library image (2 MiB per device that loads the
+ * library, held until the process exits).
+ *   - limit: B * T <= confu_tree_accept_static_max_rows() (4096); beyond it CONFU_ERR_WORKSPACE;
+ *   - the first call on a device looks the array's device address up (one runtime query, no
+ *     allocation) with the current device; make that first call outside any stream capture;
+ *   - all calls share the array and it keeps the last call's contents (nothing in it needs
+ *     clearing: a call only reads what its own first kernel wrote); calls that overlap on the GPU
+ *     race on it, so run them one after another (one stream, or ordered streams);
+ *   - the call uses the current device; all pointers are device pointers of that device.
+ */
+size_t confu_tree_accept_static_max_rows(void);
+int confu_tree_accept_static(int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
+                             const void* target_logits, const void* draft_logits,
+                             const int32_t* tokens, const int32_t* parent, const int32_t* con_owner,
+                             const float* uniforms, float temperature, int32_t sibling_mode,
+                             int32_t* accept_len, int32_t* path, int32_t* next_token, int32_t* future_row,
+                             int32_t* counters, int32_t* status, void* stream);
+
 /* ---- KV compaction (Sec. 2 step 4: the accepted sequence is the next input) ---- */
 
 /*

@@ -21,6 +21,7 @@ EXPORTS = [
     "confu_create", "confu_destroy", "confu_workspace_bytes", "confu_set_workspace", "confu_status_string",
     "confu_last_cuda_error", "confu_plan_bytes", "confu_tree_plan", "confu_tree_attention",
     "confu_accept_workspace_bytes", "confu_tree_accept", "confu_kv_compact", "confu_kv_append",
+    "confu_tree_accept_static_max_rows", "confu_tree_accept_static",
 ]
 
 
@@ -43,10 +44,11 @@ def lib():
         L.confu_workspace_bytes.restype = C.c_size_t
         L.confu_plan_bytes.restype = C.c_size_t
         L.confu_accept_workspace_bytes.restype = C.c_size_t
+        L.confu_tree_accept_static_max_rows.restype = C.c_size_t
         L.confu_status_string.restype = C.c_char_p
         L.confu_last_cuda_error.restype = C.c_char_p
         for n in ("confu_create", "confu_destroy", "confu_set_workspace", "confu_tree_plan", "confu_tree_attention",
-                  "confu_tree_accept", "confu_kv_compact", "confu_kv_append"):
+                  "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -141,6 +143,24 @@ def confu_tree_accept(ctx, B, T, Cn, V, logit_dtype, target_logits, draft_logits
                                    C.c_float(temperature), C.c_int32(sibling_mode), _ptr(accept_len), _ptr(path),
                                    _ptr(next_token), _ptr(future_row), _ptr(counters), _ptr(workspace),
                                    C.c_size_t(ws_bytes), _ptr(status), _stream(stream)), ctx)
+
+
+def confu_tree_accept_static_max_rows():
+    return int(lib().confu_tree_accept_static_max_rows())
+
+
+def confu_tree_accept_static(B, T, Cn, V, logit_dtype, target_logits, draft_logits, tokens, parent, con_owner,
+                             uniforms, temperature, sibling_mode, accept_len, path, next_token, future_row, counters,
+                             status, stream=None):
+    """confu_tree_accept for callers that may not allocate: no context, no workspace (the library's
+    fixed scratch is used; B * T is limited to confu_tree_accept_static_max_rows())."""
+    _check("confu_tree_accept_static",
+           lib().confu_tree_accept_static(C.c_int32(B), C.c_int32(T), C.c_int32(Cn), C.c_int32(V),
+                                          C.c_int32(dtype_code(logit_dtype)), _ptr(target_logits),
+                                          _ptr(draft_logits), _ptr(tokens), _ptr(parent), _ptr(con_owner),
+                                          _ptr(uniforms), C.c_float(temperature), C.c_int32(sibling_mode),
+                                          _ptr(accept_len), _ptr(path), _ptr(next_token), _ptr(future_row),
+                                          _ptr(counters), _ptr(status), _stream(stream)))
 
 
 def confu_kv_compact(ctx, dims, n_layers, k_layer_ptrs, v_layer_ptrs, seq_start, prefix_len, accept_len, path,
