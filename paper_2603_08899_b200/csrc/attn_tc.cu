@@ -6,17 +6,21 @@
 // head: two M tiles of 128 rows (32 rows x G heads each, padded when G < 4).  Per key tile:
 //     S_t = Q_t K^T           tcgen05.mma, A and B from shared memory (K-major, 128B swizzle)
 //     P_t = exp2(S_t*c - m)   one thread per row: tcgen05.ld, mask (last tiles only), tcgen05.st as bf16
+//                             over the S columns, handed over in two halves of 64 keys
 //     O_t += P_t V            tcgen05.mma, A from TMEM, B = V tile in shared memory (MN-major)
-// The two M tiles ping-pong: while the softmax warps of one tile work, the tensor pipe runs the
-// other tile's MMAs.  Prefix tiles need no mask; the ancestor bitmask (one 64-bit word per row,
-// in a register) is applied only to the tiles that hold the tree slots, the ragged tail and the
-// soft-prompt entries.  A range that does not cover a whole pair writes an unnormalised partial
-// (O, m, l) that combine_kernel merges in a fixed order.
+// Each M tile has its own softmax warpgroup; the two run out of phase, so that while one computes
+// exponentials the tensor pipe serves the other (P V of the half that is ready, then the next
+// Q K^T).  Prefix tiles need no mask; the ancestor bitmask (one 64-bit word per row, in a register) is applied only to
+// the tiles that hold the tree slots, the ragged tail and the soft-prompt entries.  A range that
+// does not cover a whole pair writes an unnormalised partial (O, m, l) that combine_kernel merges
+// in a fixed order.
 //
 // Every wait on an mbarrier is bounded (wall-clock limit); on expiry the CTA raises an abort flag,
 // every role leaves its loop, tensor memory is released and CONFU_ST_TIMEOUT is reported.
 #include <cuda.h>
 #include <stdlib.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -24,13 +28,14 @@ namespace confu {
 
 namespace tc {
 
-constexpr int kThreads = 384;            // warps 0-3: softmax tile 0, 4-7: softmax tile 1, 8: TMA, 9: MMA
+constexpr int kThreads = 384;            // warps 0-3: softmax of M tile 0, 4-7: of M tile 1, 8: TMA, 9: MMA
 constexpr int kStages = 4;               // ring of 32 KB slots shared by K and V tiles
 constexpr int kD = 128;
 constexpr int kTileBytes = kTileKeys * kD * 2;      // 32 KB
 constexpr int kHalfTile = kTileBytes / 2;           // one 64-wide half of the head dim: [128 rows][128 B]
 constexpr int kQBytes = 2 * kTileBytes;             // two M tiles
 constexpr uint32_t kTmemCols = 512;                 // S0 | S1 | O0 | O1, 128 columns each; P_t overlays S_t
+constexpr int kPolyPeriod = 4, kPolyCount = 0;      // of every kPolyPeriod element pairs, kPolyCount take the polynomial 2^x
 constexpr float kRescaleThreshold = 8.f;            // lazy rescale: move the reference max only past 2^8
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -39,7 +44,7 @@ struct SharedStorage {
     alignas(1024) uint8_t kv[kStages][kTileBytes];
     alignas(8) uint64_t q_full, q_empty;
     uint64_t kv_full[kStages], kv_empty[kStages];
-    uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
+    uint64_t s_full[2], p_full[2][2], o_done[2];     // p_full[M tile][key half]
     uint32_t tmem_base;
     int abort;
 };
@@ -113,6 +118,9 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
         : "memory");
 }
 
+// high word of every shared-memory descriptor: SBO = 1024 B (>> 4) | version 1 (bit 46) | swizzle 128B (code 2, bits 61-63)
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -123,25 +131,29 @@ __device__ __forceinline__ void tc_commit(uint64_t* bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
 }
+// Shared-memory matrix descriptors are passed as their two 32-bit words: the low word carries the
+// start address and the leading byte offset (both >> 4), the high word is the same for every
+// operand of this kernel (stride byte offset 1024, descriptor version 1, 128-byte swizzle).
 // D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc)
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(acc), "r"(kDescHi)
         : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc)
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "mov.b64 db, {%2, %5};\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(acc), "r"(kDescHi)
         : "memory");
 }
-
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 {
     asm volatile(
@@ -174,6 +186,47 @@ __device__ __forceinline__ float ex2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Packed fp32 pairs (one 64-bit register): the FMA pipe takes two lanes per instruction.
+__device__ __forceinline__ uint64_t f2_pack(float a, float b)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// 2^x for two finite x <= ~8 on the FMA and integer pipes, leaving the MUFU to the other elements:
+// x = j + f with j = round(x), f in [-0.5, 0.5]; 2^f by a cubic (relative error 7.6e-5, far below
+// the bf16 rounding of P); 2^j by adding j to the exponent field.  x is clamped at -125.
+__device__ __forceinline__ void exp2_poly2(float x0, float x1, float& y0, float& y1)
+{
+    const float kMagic = 12582912.f;                          // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
+    const uint64_t xc = f2_pack(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
+    const uint64_t t = f2_add(xc, f2_pack(kMagic, kMagic));
+    const uint64_t jf = f2_add(t, f2_pack(-kMagic, -kMagic));
+    const uint64_t f = f2_fma(jf, f2_pack(-1.f, -1.f), xc);
+    uint64_t p = f2_fma(f, f2_pack(0.05520550534129143f, 0.05520550534129143f), f2_pack(0.24261397123336792f, 0.24261397123336792f));
+    p = f2_fma(p, f, f2_pack(0.6932547688484192f, 0.6932547688484192f));
+    p = f2_fma(p, f, f2_pack(0.9999276995658875f, 0.9999276995658875f));
+    float p0, p1, t0, t1;
+    f2_unpack(p, p0, p1);
+    f2_unpack(t, t0, t1);
+    y0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+    y1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     uint32_t r;
@@ -181,13 +234,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return r;
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle (layout code 2), descriptor version 1.
-// lbo / sbo in bytes: leading / stride byte offsets of the canonical layout.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
-{
-    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
-           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
-}
+// Low word of a shared-memory matrix descriptor: start address and leading byte offset, both >> 4.
+// K-major operands (Q, K) ignore the leading offset (16 B by convention); the MN-major V tile uses
+// it as the distance between its two 64-column halves.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo) { return ((addr >> 4) & 0x3FFFu) | ((lbo >> 4) << 16); }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; B K-major (QK^T) or MN-major (PV).
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
@@ -274,47 +324,62 @@ __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanVi
     }
 }
 
+// The MMA warp runs this loop with all 32 lanes converged, so that every value an instruction
+// descriptor is built from is warp-uniform; only the tcgen05 instructions themselves are
+// predicated on the elected lane.  kTwo: both M tiles are in use (R > 32).
+template <bool kTwo>
 __device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem)
 {
+    constexpr int kMt = kTwo ? 2 : 1;
+    const bool el = (threadIdx.x & 31) == 0;
     Walker w(pv, prm, blockIdx.x);
     Segment s;
     uint32_t ring = 0, seg = 0;
-    uint32_t n_s[2] = {0, 0};          // S tiles produced per M tile (phase of s_full)
-    uint32_t n_p[2] = {0, 0};          // P tiles consumed per M tile (phase of p_full)
-    const uint32_t q_addr = smem_u32(sh.q);
+    uint32_t n_p = 0;                  // key tiles whose P has been consumed (phase of the p_full barriers)
+    // descriptor low words: Q tiles (K-major); ring slot i seen as a K tile (K-major) or as a V
+    // tile (MN-major, its two 64-column halves kHalfTile apart) = slot 0's word + i * slot size
+    const uint32_t q_lo = desc_lo(smem_u32(sh.q), 16);
+    const uint32_t k_lo0 = desc_lo(smem_u32(sh.kv[0]), 16), v_lo0 = desc_lo(smem_u32(sh.kv[0]), kHalfTile);
+    constexpr uint32_t kSlotStep = kTileBytes >> 4;
 
-    auto issue_qk = [&](int t, uint32_t k_addr) {
+    // S_t = Q_t K^T: 8 steps of 16 head dims; step i sits in 64-column half i/4 at byte 32*(i%4) of the swizzled row
+    auto issue_qk = [&](int t, uint32_t kl) {
+        if (el) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t off = (uint32_t)(i >> 2) * kHalfTile + (uint32_t)(i & 3) * 32u;
-            mma_ss(tmem + t * 128, smem_desc(q_addr + t * kTileBytes + off, 16, 1024),
-                   smem_desc(k_addr + off, 16, 1024), kIdescQK, i > 0 ? 1u : 0u);
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t off = ((uint32_t)(i >> 2) * kHalfTile + (uint32_t)(i & 3) * 32u) >> 4;
+                mma_ss(tmem + t * 128, q_lo + t * kSlotStep + off, kl + off, kIdescQK, i > 0 ? 1u : 0u);
+            }
+            tc_commit(&sh.s_full[t]);
         }
-        tc_commit(&sh.s_full[t]);
-        ++n_s[t];
     };
-    auto issue_pv = [&](int t, uint32_t v_addr, bool first_of_segment) {
+    // O_t += P_t V for one half of the key tile: 4 steps of 16 keys (2048 B of the V tile and 8
+    // TMEM columns of bf16 pairs each); P sits in the first 64 columns of the S_t block
+    auto issue_pv = [&](int t, int half, uint32_t vl, bool first_of_segment) {
+        if (el) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
-            mma_ts(tmem + 256 + t * 128, tmem + t * 128 + i * 8, smem_desc(v_addr + i * 2048u, kHalfTile, 1024), kIdescPV,
-                   (first_of_segment && i == 0) ? 0u : 1u);
+            for (int k = 0; k < 4; ++k) {
+                const int i = 4 * half + k;
+                mma_ts(tmem + 256 + t * 128, tmem + t * 128 + i * 8, vl + i * (2048u >> 4), kIdescPV,
+                       (first_of_segment && i == 0) ? 0u : 1u);
+            }
+        }
     };
 
     while (w.next(s)) {
         const int n_tiles = s.t1 - s.t0;
         if (!mbar_wait(&sh.q_full, seg & 1, &sh.abort)) return;
-        // accumulators of the previous pair must have been read out
-        for (int t = 0; t < prm.n_mt; ++t)
-            if (!mbar_wait(&sh.o_free[t], (seg & 1) ^ 1, &sh.abort)) return;
-        tc_fence_after();
-        // first key tile: S_0, S_1
+        // first key tile: S_0, S_1.  (The first P V below overwrites the previous pair's O_t; the
+        // softmax threads hand P over only after they have read that O_t out, so waiting for P
+        // orders the two.)
         uint32_t k_slot = ring % kStages;
         if (!mbar_wait(&sh.kv_full[k_slot], (ring / kStages) & 1, &sh.abort)) return;
         tc_fence_after();
-        for (int t = 0; t < prm.n_mt; ++t) issue_qk(t, smem_u32(sh.kv[k_slot]));
-        tc_commit(&sh.kv_empty[k_slot]);
+#pragma unroll
+        for (int t = 0; t < kMt; ++t) issue_qk(t, k_lo0 + k_slot * kSlotStep);
+        if (el) tc_commit(&sh.kv_empty[k_slot]);
         ++ring;
-        if (n_tiles == 1) tc_commit(&sh.q_empty);
+        if (n_tiles == 1 && el) tc_commit(&sh.q_empty);
         for (int j = 0; j < n_tiles; ++j) {
             const uint32_t v_slot = ring % kStages;
             if (!mbar_wait(&sh.kv_full[v_slot], (ring / kStages) & 1, &sh.abort)) return;
@@ -326,18 +391,25 @@ __device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& p
                 if (!mbar_wait(&sh.kv_full[nk_slot], (ring / kStages) & 1, &sh.abort)) return;
                 ++ring;
             }
-            for (int t = 0; t < prm.n_mt; ++t) {
-                if (!mbar_wait(&sh.p_full[t], n_p[t] & 1, &sh.abort)) return;
-                ++n_p[t];
+            const uint32_t vl = v_lo0 + v_slot * kSlotStep, kl = k_lo0 + nk_slot * kSlotStep;
+#pragma unroll
+            for (int t = 0; t < kMt; ++t) {
+                if (!mbar_wait(&sh.p_full[t][0], n_p & 1, &sh.abort)) return;
                 tc_fence_after();
-                issue_pv(t, smem_u32(sh.kv[v_slot]), j == 0);
-                if (!more) tc_commit(&sh.o_done[t]);
-                if (more) issue_qk(t, smem_u32(sh.kv[nk_slot]));
+                issue_pv(t, 0, vl, j == 0);
+                if (!mbar_wait(&sh.p_full[t][1], n_p & 1, &sh.abort)) return;
+                tc_fence_after();
+                issue_pv(t, 1, vl, false);
+                if (more) issue_qk(t, kl);
+                else if (el) tc_commit(&sh.o_done[t]);
             }
-            tc_commit(&sh.kv_empty[v_slot]);
-            if (more) {
-                tc_commit(&sh.kv_empty[nk_slot]);
-                if (j + 2 == n_tiles) tc_commit(&sh.q_empty);       // last QK of the pair has been issued
+            ++n_p;
+            if (el) {
+                tc_commit(&sh.kv_empty[v_slot]);
+                if (more) {
+                    tc_commit(&sh.kv_empty[nk_slot]);
+                    if (j + 2 == n_tiles) tc_commit(&sh.q_empty);       // last QK of the pair has been issued
+                }
             }
         }
         ++seg;
@@ -366,6 +438,40 @@ __device__ __forceinline__ void visible_bits(const Segment& s, int t, int R, int
     else if (off > -64) v |= m >> (-off);
     lo = (uint64_t)v;
     hi = (uint64_t)(v >> 64);
+}
+
+// max of 128 floats held as raw bits, as eight independent chains of three-input max
+__device__ __forceinline__ float max128(const uint32_t (&sv)[128])
+{
+    float a[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        a[k] = fmaxf(__uint_as_float(sv[16 * k]), __uint_as_float(sv[16 * k + 1]));
+#pragma unroll
+        for (int j = 2; j < 16; j += 2)
+            asm("max.f32 %0, %0, %1, %2;" : "+f"(a[k]) : "f"(__uint_as_float(sv[16 * k + j])), "f"(__uint_as_float(sv[16 * k + j + 1])));
+    }
+    return fmaxf(fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3])), fmaxf(fmaxf(a[4], a[5]), fmaxf(a[6], a[7])));
+}
+
+// exp2(s*c - m) of 64 scores -> 32 packed bf16 pairs; returns their fp32 sum
+template <bool kUsePoly>
+__device__ __forceinline__ float weights64(const uint32_t* sv, float c, float neg_m, uint32_t (&pk)[32])
+{
+    uint64_t sum2 = f2_pack(0.f, 0.f);
+    const uint64_t c2 = f2_pack(c, c), nm2 = f2_pack(neg_m, neg_m);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        float x0, x1, p0, p1;
+        f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1])), c2, nm2), x0, x1);
+        if (kUsePoly && (j % kPolyPeriod) < kPolyCount) exp2_poly2(x0, x1, p0, p1);
+        else { p0 = ex2(x0); p1 = ex2(x1); }
+        sum2 = f2_add(sum2, f2_pack(p0, p1));
+        pk[j] = pack_bf16(p0, p1);
+    }
+    float s0, s1;
+    f2_unpack(sum2, s0, s1);
+    return s0 + s1;
 }
 
 __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem, int t /*M tile*/)
@@ -404,10 +510,7 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
                     if (!((hi >> j) & 1ull)) sv[64 + j] = 0xff800000u;
                 }
             }
-            float mx = __uint_as_float(sv[0]);
-#pragma unroll
-            for (int j = 1; j < 128; ++j) mx = fmaxf(mx, __uint_as_float(sv[j]));
-            const float m_new = fmaxf(m_ref, mx * c);
+            const float m_new = fmaxf(m_ref, max128(sv) * c);
             if (tile == s.t0) {
                 m_ref = m_new;
             } else {
@@ -428,21 +531,18 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
                 }
             }
             const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-            float sum = 0.f;
-            uint32_t pk[64];
+            // The two halves of P go to the tensor pipe as soon as each is stored: P V of keys 0-63
+            // runs while the exponentials of keys 64-127 are computed.  Masked tiles hold -inf
+            // scores, whose weight must be exactly 0: there every element takes the MUFU.
 #pragma unroll
-            for (int j = 0; j < 64; ++j) {
-                const float p0 = ex2(fmaf(__uint_as_float(sv[2 * j]), c, neg_m));
-                const float p1 = ex2(fmaf(__uint_as_float(sv[2 * j + 1]), c, neg_m));
-                sum += p0 + p1;
-                pk[j] = pack_bf16(p0, p1);
+            for (int half = 0; half < 2; ++half) {
+                uint32_t pk[32];
+                l += masked ? weights64<false>(&sv[64 * half], c, neg_m, pk) : weights64<true>(&sv[64 * half], c, neg_m, pk);
+                tmem_st32(s_addr + 32 * half, pk);
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(&sh.p_full[t][half]);
             }
-            l += sum;
-            tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-            tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(&sh.p_full[t]);
         }
         // ---- epilogue of this pair / range ----
         if (!mbar_wait(&sh.o_done[t], seg & 1, &sh.abort)) return;
@@ -486,8 +586,9 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
             ml[t * 128 + lane_row] = m_ref;
             ml[kPartRows + t * 128 + lane_row] = l;
         }
+        // the P of the next range's first tile is only handed over after this point, which is what
+        // keeps the tensor pipe from overwriting O_t before it has been read
         tc_fence_before();
-        mbar_arrive(&sh.o_free[t]);
         ++seg;
     }
 }
@@ -509,9 +610,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&sh.s_full[t], 1);
-            mbar_init(&sh.p_full[t], 128);
+            mbar_init(&sh.p_full[t][0], 128);
+            mbar_init(&sh.p_full[t][1], 128);
             mbar_init(&sh.o_done[t], 1);
-            mbar_init(&sh.o_free[t], 128);
         }
         sh.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -537,7 +638,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         if (warp == 8) {
             if ((threadIdx.x & 31) == 0) producer_role(sh, prm, pv, &q_map, &k_map, &v_map, &ks_map, &vs_map);
         } else if (warp == 9) {
-            if ((threadIdx.x & 31) == 0) mma_role(sh, prm, pv, tmem);
+            if (prm.n_mt > 1) mma_role<true>(sh, prm, pv, tmem);
+            else mma_role<false>(sh, prm, pv, tmem);
         }
         __syncwarp();
     }
