@@ -254,7 +254,7 @@ struct Segment {
 
 struct Walker {
     const PlanView pv;
-    int64_t f, f1;
+    int64_t f, f1;             // this CTA's share of the cost line: positions [f, f1)
     int cta;
     const Params& prm;
     __device__ Walker(const PlanView& v, const Params& p, int cta_) : pv(v), cta(cta_), prm(p)
@@ -264,28 +264,38 @@ struct Walker {
         f = (int64_t)cta_ * N / n;
         f1 = (int64_t)(cta_ + 1) * N / n;
     }
+    // Next non-empty run of key tiles of one pair inside the share; false when the share is used up.
     __device__ bool next(Segment& s)
     {
-        if (f >= f1) return false;
-        int lo = 0, hi = prm.d.B;                  // largest b with tile_base[b] <= f
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (pv.tile_base[mid] <= f) lo = mid; else hi = mid;
+        while (f < f1) {
+            int lo = 0, hi = prm.d.B;                  // largest b with tile_base[b] <= f
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (pv.tile_base[mid] <= f) lo = mid; else hi = mid;
+            }
+            const int nt = pv.tiles[lo];
+            const int cost = nt + kPairOverheadTiles;
+            const int64_t local = f - pv.tile_base[lo];
+            const int pos = (int)(local % cost);
+            const int64_t room = f1 - f;
+            const int take = (int)((int64_t)(cost - pos) <= room ? cost - pos : room);
+            f += take;
+            const int t0 = pos > kPairOverheadTiles ? pos - kPairOverheadTiles : 0;
+            const int t1 = pos + take > kPairOverheadTiles ? pos + take - kPairOverheadTiles : 0;
+            if (t1 <= t0) continue;                    // the share ended inside this pair's overhead zone
+            s.b = lo;
+            s.nt = nt;
+            s.g = (int)(local / cost);
+            s.t0 = t0;
+            s.t1 = t1;
+            s.nkt = nt - (prm.d.S > 0 ? 1 : 0);
+            s.P = prm.prefix_len[lo];
+            s.slot0 = prm.seq_start[lo];
+            const bool whole = t0 == 0 && t1 == nt;
+            s.part_slot = whole ? -1 : 2 * cta + (t1 < nt ? 1 : 0);
+            return true;
         }
-        s.b = lo;
-        s.nt = pv.tiles[lo];
-        const int64_t local = f - pv.tile_base[lo];
-        s.g = (int)(local / s.nt);
-        s.t0 = (int)(local % s.nt);
-        const int64_t room = f1 - f;
-        s.t1 = (int)((int64_t)(s.nt - s.t0) <= room ? s.nt : s.t0 + room);
-        s.nkt = s.nt - (prm.d.S > 0 ? 1 : 0);
-        s.P = prm.prefix_len[lo];
-        s.slot0 = prm.seq_start[lo];
-        const bool whole = s.t0 == 0 && s.t1 == s.nt;
-        s.part_slot = whole ? -1 : 2 * cta + (s.t1 < s.nt ? 1 : 0);
-        f += s.t1 - s.t0;
-        return true;
+        return false;
     }
 };
 
@@ -661,7 +671,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 }
 
 // Merge of the split-KV partials of one (sequence, kv head) pair, in CTA order (deterministic).
-__global__ void __launch_bounds__(128) combine_kernel(const Params prm)
+// One block per (pair, M tile); a warp takes a row at a time, lane i the row's columns 4i..4i+3, so
+// partial rows are read and output rows written as whole 512- and 256-byte lines.
+__global__ void __launch_bounds__(256) combine_kernel(const Params prm)
 {
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
     const int pair = blockIdx.x, t = blockIdx.y;
@@ -669,49 +681,41 @@ __global__ void __launch_bounds__(128) combine_kernel(const Params prm)
     const int nt = pv.tiles[b];
     if (nt == 0 || t >= prm.n_mt) return;
     const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
-    const int64_t F = pv.tile_base[b] + (int64_t)g * nt;
+    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
+    const int64_t F = pv.tile_base[b] + (int64_t)g * (nt + kPairOverheadTiles) + kPairOverheadTiles;
     const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
     if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
     const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
-    const int lane_row = threadIdx.x;
-    const int r = 32 * t + lane_row / G, hl = lane_row % G;
-    if (!(lane_row < 32 * G && r < R)) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t slot_floats = partial_slot_bytes() / sizeof(float);
-    const int row = t * 128 + lane_row;
-    float M = -INFINITY;
-    for (int cta = c_first; cta <= c_last; ++cta) {
-        const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
-        M = fmaxf(M, slot[(size_t)kPartRows * kPartD + row]);
-    }
-    float acc[kPartD];
-#pragma unroll
-    for (int j = 0; j < kPartD; ++j) acc[j] = 0.f;
-    float L = 0.f;
-    for (int cta = c_first; cta <= c_last; ++cta) {
-        const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
-        const float m = slot[(size_t)kPartRows * kPartD + row];
-        const float w = (m == -INFINITY) ? 0.f : ex2(m - M);
-        L += w * slot[(size_t)kPartRows * kPartD + kPartRows + row];
-        const float4* prow = reinterpret_cast<const float4*>(slot + (size_t)row * kPartD);
-#pragma unroll
-        for (int j = 0; j < kPartD / 4; ++j) {
-            const float4 v = prow[j];
-            acc[4 * j] += w * v.x; acc[4 * j + 1] += w * v.y; acc[4 * j + 2] += w * v.z; acc[4 * j + 3] += w * v.w;
+    for (int lane_row = warp; lane_row < 32 * G; lane_row += 8) {
+        const int r = 32 * t + lane_row / G, hl = lane_row % G;
+        if (r >= R) break;
+        const int row = t * 128 + lane_row;
+        float M = -INFINITY;
+        for (int cta = c_first; cta <= c_last; ++cta) {
+            const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
+            M = fmaxf(M, slot[(size_t)kPartRows * kPartD + row]);
         }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float L = 0.f;
+        for (int cta = c_first; cta <= c_last; ++cta) {
+            const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
+            const float m = slot[(size_t)kPartRows * kPartD + row];
+            const float w = (m == -INFINITY) ? 0.f : ex2(m - M);
+            L += w * slot[(size_t)kPartRows * kPartD + kPartRows + row];
+            const float4 v = reinterpret_cast<const float4*>(slot + (size_t)row * kPartD)[lane];
+            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+        }
+        const float inv_l = 1.f / L;
+        const int h = g * G + hl;
+        __nv_bfloat16* orow = prm.out + (((size_t)b * R + r) * Hq + h) * kD;
+        uint2 pkt;
+        pkt.x = pack_bf16(acc.x * inv_l, acc.y * inv_l);
+        pkt.y = pack_bf16(acc.z * inv_l, acc.w * inv_l);
+        reinterpret_cast<uint2*>(orow)[lane] = pkt;
+        if (prm.lse && lane == 0) prm.lse[((size_t)b * R + r) * Hq + h] = (M + log2f(L)) * 0.6931471805599453f;
     }
-    const float inv_l = 1.f / L;
-    const int h = g * G + hl;
-    __nv_bfloat16* orow = prm.out + (((size_t)b * R + r) * Hq + h) * kD;
-#pragma unroll
-    for (int j = 0; j < kPartD / 8; ++j) {
-        uint4 pkt;
-        pkt.x = pack_bf16(acc[8 * j] * inv_l, acc[8 * j + 1] * inv_l);
-        pkt.y = pack_bf16(acc[8 * j + 2] * inv_l, acc[8 * j + 3] * inv_l);
-        pkt.z = pack_bf16(acc[8 * j + 4] * inv_l, acc[8 * j + 5] * inv_l);
-        pkt.w = pack_bf16(acc[8 * j + 6] * inv_l, acc[8 * j + 7] * inv_l);
-        *reinterpret_cast<uint4*>(orow + j * 8) = pkt;
-    }
-    if (prm.lse) prm.lse[((size_t)b * R + r) * Hq + h] = (M + log2f(L)) * 0.6931471805599453f;
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -792,7 +796,7 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     attention_tc_kernel<<<ctx->sm_count, kThreads, smem, st>>>(q_map, k_map, v_map, ks_map, vs_map, prm);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    combine_kernel<<<dim3(d.B * d.Hkv, prm.n_mt), 128, 0, st>>>(prm);
+    combine_kernel<<<dim3(d.B * d.Hkv, prm.n_mt), 256, 0, st>>>(prm);
     return cudaGetLastError();
 }
 

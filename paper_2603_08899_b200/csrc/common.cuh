@@ -19,13 +19,20 @@ constexpr int kTileKeys = 128;                  // keys per attention tile (tens
 //   uint64 mask[B][64]        bit j of mask[b][r]: row r sees tree slot j
 //   int32  bad[B]             non-zero: malformed tree, sequence skipped
 //   int32  tiles[B]           key tiles of one (sequence, kv head) pair, soft-prompt tile included
-//   int64  tile_base[B + 1]   flat index of the first tile of sequence b (all Hkv heads), exclusive scan
+//   int64  tile_base[B + 1]   position of sequence b's first pair on the flat cost line (exclusive scan)
+//
+// The split-KV work is balanced on a "cost line": every (sequence, kv head) pair takes
+// tiles + kPairOverheadTiles consecutive positions (the overhead stands for loading Q, draining
+// the pipeline and writing the output once per pair), pairs in (sequence, head) order.  CTA c of n
+// gets positions [c*N/n, (c+1)*N/n); position q of a pair means key tile q - kPairOverheadTiles,
+// so a CTA whose share ends inside a pair's overhead zone takes none of its tiles.
 // ---------------------------------------------------------------------------
+constexpr int kPairOverheadTiles = 4;
 struct PlanHeader {
     int32_t B, Hkv, T, C, S, R;
     int32_t n_ctas;            // CTAs of the tensor-core attention launch (<= SM count)
     int32_t pad;
-    int64_t n_tiles;           // total tiles over all (sequence, kv head) pairs
+    int64_t n_tiles;           // length N of the cost line
 };
 
 struct PlanView {

@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
         int64_t acc = 0;
         for (int b = 0; b < B; ++b) {
             pv.tile_base[b] = acc;
-            acc += (int64_t)pv.tiles[b] * d.Hkv;
+            if (pv.tiles[b] > 0) acc += (int64_t)(pv.tiles[b] + kPairOverheadTiles) * d.Hkv;
         }
         pv.tile_base[B] = acc;
         PlanHeader h;
