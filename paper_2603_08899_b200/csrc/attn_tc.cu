@@ -6,11 +6,14 @@
 // head: two M tiles of 128 rows (32 rows x G heads each, padded when G < 4).  Per key tile:
 //     S_t = Q_t K^T           tcgen05.mma, A and B from shared memory (K-major, 128B swizzle)
 //     P_t = exp2(S_t*c - m)   one thread per row: tcgen05.ld, mask (last tiles only), tcgen05.st as bf16
-//                             over the S columns, handed over in two halves of 64 keys
+//                             over the S columns
 //     O_t += P_t V            tcgen05.mma, A from TMEM, B = V tile in shared memory (MN-major)
 // Each M tile has its own softmax warpgroup; the two run out of phase, so that while one computes
-// exponentials the tensor pipe serves the other (P V of the half that is ready, then the next
-// Q K^T).  Prefix tiles need no mask; the ancestor bitmask (one 64-bit word per row, in a register) is applied only to
+// exponentials the tensor pipe serves the other (P V, then the next Q K^T).  The tensor pipe holds
+// about one instruction ahead of the issuing thread, so whatever that thread does between MMAs is
+// idle pipe time: K/V travel in stages of [V of key tile g-1 | K of key tile g] with one full and
+// one empty barrier each, which leaves the issuing thread three waits and three commits per key
+// tile.  Prefix tiles need no mask; the ancestor bitmask (one 64-bit word per row, in a register) is applied only to
 // the tiles that hold the tree slots, the ragged tail and the soft-prompt entries.  A range that
 // does not cover a whole pair writes an unnormalised partial (O, m, l) that combine_kernel merges
 // in a fixed order.
@@ -20,8 +23,6 @@
 #include <cuda.h>
 #include <stdlib.h>
 
-#include <type_traits>
-
 #include "common.cuh"
 
 namespace confu {
@@ -29,22 +30,21 @@ namespace confu {
 namespace tc {
 
 constexpr int kThreads = 384;            // warps 0-3: softmax of M tile 0, 4-7: of M tile 1, 8: TMA, 9: MMA
-constexpr int kStages = 4;               // ring of 32 KB slots shared by K and V tiles
+constexpr int kStages = 2;               // ring of stages; stage g = [V of the CTA's g-1st key tile | K of its g-th]
 constexpr int kD = 128;
 constexpr int kTileBytes = kTileKeys * kD * 2;      // 32 KB
 constexpr int kHalfTile = kTileBytes / 2;           // one 64-wide half of the head dim: [128 rows][128 B]
 constexpr int kQBytes = 2 * kTileBytes;             // two M tiles
 constexpr uint32_t kTmemCols = 512;                 // S0 | S1 | O0 | O1, 128 columns each; P_t overlays S_t
-constexpr int kPolyPeriod = 4, kPolyCount = 0;      // of every kPolyPeriod element pairs, kPolyCount take the polynomial 2^x
 constexpr float kRescaleThreshold = 8.f;            // lazy rescale: move the reference max only past 2^8
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct SharedStorage {
     alignas(1024) uint8_t q[kQBytes];
-    alignas(1024) uint8_t kv[kStages][kTileBytes];
+    alignas(1024) uint8_t kv[kStages][2][kTileBytes];    // [stage][0: V tile, 1: K tile]
     alignas(8) uint64_t q_full, q_empty;
     uint64_t kv_full[kStages], kv_empty[kStages];
-    uint64_t s_full[2], p_full[2][2], o_done[2];     // p_full[M tile][key half]
+    uint64_t s_full[2], p_full[2], o_done[2];
     uint32_t tmem_base;
     int abort;
 };
@@ -207,26 +207,6 @@ __device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
     return r;
 }
 
-// 2^x for two finite x <= ~8 on the FMA and integer pipes, leaving the MUFU to the other elements:
-// x = j + f with j = round(x), f in [-0.5, 0.5]; 2^f by a cubic (relative error 7.6e-5, far below
-// the bf16 rounding of P); 2^j by adding j to the exponent field.  x is clamped at -125.
-__device__ __forceinline__ void exp2_poly2(float x0, float x1, float& y0, float& y1)
-{
-    const float kMagic = 12582912.f;                          // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
-    const uint64_t xc = f2_pack(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
-    const uint64_t t = f2_add(xc, f2_pack(kMagic, kMagic));
-    const uint64_t jf = f2_add(t, f2_pack(-kMagic, -kMagic));
-    const uint64_t f = f2_fma(jf, f2_pack(-1.f, -1.f), xc);
-    uint64_t p = f2_fma(f, f2_pack(0.05520550534129143f, 0.05520550534129143f), f2_pack(0.24261397123336792f, 0.24261397123336792f));
-    p = f2_fma(p, f, f2_pack(0.6932547688484192f, 0.6932547688484192f));
-    p = f2_fma(p, f, f2_pack(0.9999276995658875f, 0.9999276995658875f));
-    float p0, p1, t0, t1;
-    f2_unpack(p, p0, p1);
-    f2_unpack(t, t0, t1);
-    y0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-    y1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
-}
-
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     uint32_t r;
@@ -300,130 +280,144 @@ struct Walker {
 };
 
 // ------------------------------------------------------------------------------------ roles
+// Key tiles of the CTA's share, all pairs together, are numbered g = 0..n-1 in walking order; stage
+// g of the ring carries V of tile g-1 and K of tile g (stage 0 has no V, stage n no K).
+__device__ int count_tiles(const Params& prm, const PlanView& pv)
+{
+    Walker w(pv, prm, blockIdx.x);
+    Segment s;
+    int n = 0;
+    while (w.next(s)) n += s.t1 - s.t0;
+    return n;
+}
+
+struct TileRef {                       // where a key tile's K and V come from
+    int g, z;                          // kv head, first slot (row) of the tile
+    bool soft;                         // the soft-prompt tile
+};
+
 __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanView& pv, const CUtensorMap* q_map,
                               const CUtensorMap* k_map, const CUtensorMap* v_map, const CUtensorMap* ks_map,
                               const CUtensorMap* vs_map)
 {
+    const int n_total = count_tiles(prm, pv);
     Walker w(pv, prm, blockIdx.x);
     Segment s;
-    uint32_t ring = 0;                 // running count of ring slots filled
-    uint32_t seg = 0;
+    uint32_t stage = 0, seg = 0;       // running stage / pair counters
     const int R = prm.d.T + prm.d.C;
     const uint32_t q_box_bytes = 32u * prm.G * 128u;
+    TileRef prev = {0, 0, false};
+    bool have_prev = false;
+    // fills stage `stage` with V of `prev` (if any) and K of `cur` (if any)
+    auto fill = [&](const TileRef* cur) -> bool {
+        const uint32_t st = stage % kStages;
+        if (!mbar_wait(&sh.kv_empty[st], ((stage / kStages) & 1) ^ 1, &sh.abort)) return false;
+        mbar_arrive_expect_tx(&sh.kv_full[st], (have_prev ? kTileBytes : 0) + (cur ? kTileBytes : 0));
+        if (have_prev) {
+            const CUtensorMap* m = prev.soft ? vs_map : v_map;
+            tma_load_3d(sh.kv[st][0], m, &sh.kv_full[st], 0, prev.g, prev.z);
+            tma_load_3d(sh.kv[st][0] + kHalfTile, m, &sh.kv_full[st], 64, prev.g, prev.z);
+        }
+        if (cur) {
+            const CUtensorMap* m = cur->soft ? ks_map : k_map;
+            tma_load_3d(sh.kv[st][1], m, &sh.kv_full[st], 0, cur->g, cur->z);
+            tma_load_3d(sh.kv[st][1] + kHalfTile, m, &sh.kv_full[st], 64, cur->g, cur->z);
+        }
+        ++stage;
+        return true;
+    };
     while (w.next(s)) {
-        // Q of this pair (both M tiles, two 64-wide halves each)
-        if (!mbar_wait(&sh.q_empty, (seg & 1) ^ 1, &sh.abort)) return;
-        mbar_arrive_expect_tx(&sh.q_full, 2u * prm.n_mt * q_box_bytes);
-        for (int t = 0; t < prm.n_mt; ++t)
-            for (int kb = 0; kb < 2; ++kb)
-                tma_load_3d(sh.q + (t * 2 + kb) * kHalfTile, q_map, &sh.q_full, kb * 64, s.g * prm.G, s.b * R + 32 * t);
         for (int t = s.t0; t < s.t1; ++t) {
-            const bool soft = t >= s.nkt;
-            const int z = soft ? 0 : (int)(s.slot0 + (int64_t)t * kTileKeys);
-            for (int which = 0; which < 2; ++which) {       // K then V
-                const uint32_t st = ring % kStages;
-                if (!mbar_wait(&sh.kv_empty[st], ((ring / kStages) & 1) ^ 1, &sh.abort)) return;
-                mbar_arrive_expect_tx(&sh.kv_full[st], kTileBytes);
-                const CUtensorMap* m = which == 0 ? (soft ? ks_map : k_map) : (soft ? vs_map : v_map);
-                tma_load_3d(sh.kv[st], m, &sh.kv_full[st], 0, s.g, z);
-                tma_load_3d(sh.kv[st] + kHalfTile, m, &sh.kv_full[st], 64, s.g, z);
-                ++ring;
+            TileRef cur;
+            cur.g = s.g;
+            cur.soft = t >= s.nkt;
+            cur.z = cur.soft ? 0 : (int)(s.slot0 + (int64_t)t * kTileKeys);
+            // the stage first (it carries the previous pair's last V tile, which must not wait for
+            // the Q buffer), then, at the start of a pair, its Q (both M tiles, two 64-wide halves each)
+            if (!fill(&cur)) return;
+            if (t == s.t0) {
+                if (!mbar_wait(&sh.q_empty, (seg & 1) ^ 1, &sh.abort)) return;
+                mbar_arrive_expect_tx(&sh.q_full, 2u * prm.n_mt * q_box_bytes);
+                for (int mt = 0; mt < prm.n_mt; ++mt)
+                    for (int kb = 0; kb < 2; ++kb)
+                        tma_load_3d(sh.q + (mt * 2 + kb) * kHalfTile, q_map, &sh.q_full, kb * 64, s.g * prm.G, s.b * R + 32 * mt);
             }
+            prev = cur;
+            have_prev = true;
         }
         ++seg;
     }
+    if (n_total > 0 && !fill(nullptr)) return;
 }
 
-// The MMA warp runs this loop with all 32 lanes converged, so that every value an instruction
-// descriptor is built from is warp-uniform; only the tcgen05 instructions themselves are
-// predicated on the elected lane.  kTwo: both M tiles are in use (R > 32).
+// One thread issues all tensor-core work.  Per stage g: P V of key tile g-1 for both M tiles (each
+// as soon as its P is there), Q K^T of key tile g for both, then the stage is released.
 template <bool kTwo>
 __device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem)
 {
     constexpr int kMt = kTwo ? 2 : 1;
-    const bool el = (threadIdx.x & 31) == 0;
     Walker w(pv, prm, blockIdx.x);
     Segment s;
-    uint32_t ring = 0, seg = 0;
-    uint32_t n_p = 0;                  // key tiles whose P has been consumed (phase of the p_full barriers)
-    // descriptor low words: Q tiles (K-major); ring slot i seen as a K tile (K-major) or as a V
-    // tile (MN-major, its two 64-column halves kHalfTile apart) = slot 0's word + i * slot size
+    uint32_t stage = 0, seg = 0;
+    // descriptor low words: Q tiles (K-major); a stage's K tile (K-major) and V tile (MN-major, its
+    // two 64-column halves kHalfTile apart) = stage 0's words + stage * stage size
     const uint32_t q_lo = desc_lo(smem_u32(sh.q), 16);
-    const uint32_t k_lo0 = desc_lo(smem_u32(sh.kv[0]), 16), v_lo0 = desc_lo(smem_u32(sh.kv[0]), kHalfTile);
-    constexpr uint32_t kSlotStep = kTileBytes >> 4;
+    const uint32_t v_lo0 = desc_lo(smem_u32(sh.kv[0][0]), kHalfTile), k_lo0 = desc_lo(smem_u32(sh.kv[0][1]), 16);
+    constexpr uint32_t kTileStep = kTileBytes >> 4, kStageStep = 2 * kTileStep;
 
     // S_t = Q_t K^T: 8 steps of 16 head dims; step i sits in 64-column half i/4 at byte 32*(i%4) of the swizzled row
     auto issue_qk = [&](int t, uint32_t kl) {
-        if (el) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t off = ((uint32_t)(i >> 2) * kHalfTile + (uint32_t)(i & 3) * 32u) >> 4;
-                mma_ss(tmem + t * 128, q_lo + t * kSlotStep + off, kl + off, kIdescQK, i > 0 ? 1u : 0u);
-            }
-            tc_commit(&sh.s_full[t]);
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t off = ((uint32_t)(i >> 2) * kHalfTile + (uint32_t)(i & 3) * 32u) >> 4;
+            mma_ss(tmem + t * 128, q_lo + t * kTileStep + off, kl + off, kIdescQK, i > 0 ? 1u : 0u);
         }
+        tc_commit(&sh.s_full[t]);
     };
-    // O_t += P_t V for one half of the key tile: 4 steps of 16 keys (2048 B of the V tile and 8
-    // TMEM columns of bf16 pairs each); P sits in the first 64 columns of the S_t block
-    auto issue_pv = [&](int t, int half, uint32_t vl, bool first_of_segment) {
-        if (el) {
+    // O_t += P_t V: 8 steps of 16 keys (2048 B of the V tile and 8 TMEM columns of bf16 pairs each);
+    // P sits in the first 64 columns of the S_t block
+    auto issue_pv = [&](int t, uint32_t vl, bool first_of_segment) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int i = 4 * half + k;
-                mma_ts(tmem + 256 + t * 128, tmem + t * 128 + i * 8, vl + i * (2048u >> 4), kIdescPV,
-                       (first_of_segment && i == 0) ? 0u : 1u);
+        for (int i = 0; i < 8; ++i)
+            mma_ts(tmem + 256 + t * 128, tmem + t * 128 + i * 8, vl + i * (2048u >> 4), kIdescPV,
+                   (first_of_segment && i == 0) ? 0u : 1u);
+    };
+    // one stage: P V of the previous key tile (if any), Q K^T of the current one (if any)
+    bool have_prev = false, prev_first = false, prev_last = false;
+    auto run_stage = [&](bool have_cur, bool cur_first, bool cur_last) -> bool {
+        const uint32_t st = stage % kStages;
+        if (!mbar_wait(&sh.kv_full[st], (stage / kStages) & 1, &sh.abort)) return false;
+        if (have_cur && cur_first && !mbar_wait(&sh.q_full, seg & 1, &sh.abort)) return false;
+        tc_fence_after();
+        const uint32_t vl = v_lo0 + st * kStageStep, kl = k_lo0 + st * kStageStep;
+#pragma unroll
+        for (int t = 0; t < kMt; ++t) {
+            if (have_prev) {
+                // (At the start of a pair this P V overwrites the previous pair's O_t; the softmax
+                // threads hand P over only after they have read that O_t out.)
+                if (!mbar_wait(&sh.p_full[t], (stage - 1) & 1, &sh.abort)) return false;
+                tc_fence_after();
+                issue_pv(t, vl, prev_first);
+                if (prev_last) tc_commit(&sh.o_done[t]);
             }
+            if (have_cur) issue_qk(t, kl);
         }
+        tc_commit(&sh.kv_empty[st]);
+        if (have_cur && cur_last) tc_commit(&sh.q_empty);               // last Q K^T of the pair has been issued
+        ++stage;
+        have_prev = have_cur;
+        prev_first = cur_first;
+        prev_last = cur_last;
+        return true;
     };
 
     while (w.next(s)) {
         const int n_tiles = s.t1 - s.t0;
-        if (!mbar_wait(&sh.q_full, seg & 1, &sh.abort)) return;
-        // first key tile: S_0, S_1.  (The first P V below overwrites the previous pair's O_t; the
-        // softmax threads hand P over only after they have read that O_t out, so waiting for P
-        // orders the two.)
-        uint32_t k_slot = ring % kStages;
-        if (!mbar_wait(&sh.kv_full[k_slot], (ring / kStages) & 1, &sh.abort)) return;
-        tc_fence_after();
-#pragma unroll
-        for (int t = 0; t < kMt; ++t) issue_qk(t, k_lo0 + k_slot * kSlotStep);
-        if (el) tc_commit(&sh.kv_empty[k_slot]);
-        ++ring;
-        if (n_tiles == 1 && el) tc_commit(&sh.q_empty);
-        for (int j = 0; j < n_tiles; ++j) {
-            const uint32_t v_slot = ring % kStages;
-            if (!mbar_wait(&sh.kv_full[v_slot], (ring / kStages) & 1, &sh.abort)) return;
-            ++ring;
-            const bool more = j + 1 < n_tiles;
-            uint32_t nk_slot = 0;
-            if (more) {
-                nk_slot = ring % kStages;
-                if (!mbar_wait(&sh.kv_full[nk_slot], (ring / kStages) & 1, &sh.abort)) return;
-                ++ring;
-            }
-            const uint32_t vl = v_lo0 + v_slot * kSlotStep, kl = k_lo0 + nk_slot * kSlotStep;
-#pragma unroll
-            for (int t = 0; t < kMt; ++t) {
-                if (!mbar_wait(&sh.p_full[t][0], n_p & 1, &sh.abort)) return;
-                tc_fence_after();
-                issue_pv(t, 0, vl, j == 0);
-                if (!mbar_wait(&sh.p_full[t][1], n_p & 1, &sh.abort)) return;
-                tc_fence_after();
-                issue_pv(t, 1, vl, false);
-                if (more) issue_qk(t, kl);
-                else if (el) tc_commit(&sh.o_done[t]);
-            }
-            ++n_p;
-            if (el) {
-                tc_commit(&sh.kv_empty[v_slot]);
-                if (more) {
-                    tc_commit(&sh.kv_empty[nk_slot]);
-                    if (j + 2 == n_tiles) tc_commit(&sh.q_empty);       // last QK of the pair has been issued
-                }
-            }
-        }
+        for (int j = 0; j < n_tiles; ++j)
+            if (!run_stage(true, j == 0, j + 1 == n_tiles)) return;
         ++seg;
     }
+    if (have_prev) run_stage(false, false, false);
 }
 
 // Which of the 128 keys of tile `t` may row r see.  lo: keys 0..63 of the tile, hi: 64..127.
@@ -465,17 +459,15 @@ __device__ __forceinline__ float max128(const uint32_t (&sv)[128])
 }
 
 // exp2(s*c - m) of 64 scores -> 32 packed bf16 pairs; returns their fp32 sum
-template <bool kUsePoly>
 __device__ __forceinline__ float weights64(const uint32_t* sv, float c, float neg_m, uint32_t (&pk)[32])
 {
     uint64_t sum2 = f2_pack(0.f, 0.f);
     const uint64_t c2 = f2_pack(c, c), nm2 = f2_pack(neg_m, neg_m);
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-        float x0, x1, p0, p1;
+        float x0, x1;
         f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1])), c2, nm2), x0, x1);
-        if (kUsePoly && (j % kPolyPeriod) < kPolyCount) exp2_poly2(x0, x1, p0, p1);
-        else { p0 = ex2(x0); p1 = ex2(x1); }
+        const float p0 = ex2(x0), p1 = ex2(x1);
         sum2 = f2_add(sum2, f2_pack(p0, p1));
         pk[j] = pack_bf16(p0, p1);
     }
@@ -541,18 +533,17 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
                 }
             }
             const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-            // The two halves of P go to the tensor pipe as soon as each is stored: P V of keys 0-63
-            // runs while the exponentials of keys 64-127 are computed.  Masked tiles hold -inf
-            // scores, whose weight must be exactly 0: there every element takes the MUFU.
+            // P overlays the first 64 columns of S_t (all of S_t is in registers by now); masked
+            // scores are -inf and get weight exactly 0
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t pk[32];
-                l += masked ? weights64<false>(&sv[64 * half], c, neg_m, pk) : weights64<true>(&sv[64 * half], c, neg_m, pk);
+                l += weights64(&sv[64 * half], c, neg_m, pk);
                 tmem_st32(s_addr + 32 * half, pk);
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(&sh.p_full[t][half]);
             }
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(&sh.p_full[t]);
         }
         // ---- epilogue of this pair / range ----
         if (!mbar_wait(&sh.o_done[t], seg & 1, &sh.abort)) return;
@@ -620,8 +611,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&sh.s_full[t], 1);
-            mbar_init(&sh.p_full[t][0], 128);
-            mbar_init(&sh.p_full[t][1], 128);
+            mbar_init(&sh.p_full[t], 128);
             mbar_init(&sh.o_done[t], 1);
         }
         sh.abort = 0;
@@ -648,8 +638,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
         if (warp == 8) {
             if ((threadIdx.x & 31) == 0) producer_role(sh, prm, pv, &q_map, &k_map, &v_map, &ks_map, &vs_map);
         } else if (warp == 9) {
-            if (prm.n_mt > 1) mma_role<true>(sh, prm, pv, tmem);
-            else mma_role<false>(sh, prm, pv, tmem);
+            if ((threadIdx.x & 31) == 0) {
+                if (prm.n_mt > 1) mma_role<true>(sh, prm, pv, tmem);
+                else mma_role<false>(sh, prm, pv, tmem);
+            }
         }
         __syncwarp();
     }
