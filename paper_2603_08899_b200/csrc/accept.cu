@@ -3,11 +3,15 @@
 //   row_stats_kernel   one streaming pass over every logit row of the target and draft matrices:
 //                      per row chunk the running max, the sum of exp((x - max)/temperature) (online
 //                      softmax), the lowest index of the max, and a non-finite flag.  HBM bound.
-//   accept_walk_kernel one CTA per sequence: the sequential accept / reject walk.  After the k-th
-//                      rejection at a node the target row is norm(max(p - q, 0)) applied k times;
-//                      it is never materialised: each pass re-evaluates the k-level recursion per
-//                      vocabulary entry from the two logit rows (L2 resident) and only the
-//                      normalisers Z_1..Z_k are kept.
+//   accept_walk_kernel one thread-block cluster of kWalkCluster CTAs per sequence: the sequential
+//                      accept / reject walk.  After the k-th rejection at a node the target row is
+//                      norm(max(p - q, 0)) applied k times; it is never materialised: each pass
+//                      re-evaluates the k-level recursion per vocabulary entry from the two logit
+//                      rows (L2 resident) and only the normalisers Z_1..Z_k are kept.  Every CTA of
+//                      the cluster runs the same control flow on the same data; only the passes over
+//                      the vocabulary are shared out (strip s to CTA s mod kWalkCluster), the strip
+//                      sums being written into every CTA's shared memory before a cluster barrier.
+#include <cooperative_groups.h>
 #include <limits.h>
 
 #include "common.cuh"
@@ -16,6 +20,7 @@ namespace confu {
 
 constexpr int kStatChunksMax = 16;
 constexpr int kWalkThreads = 512;
+constexpr int kWalkCluster = 8;                           // CTAs per sequence (portable cluster size)
 constexpr int kEpt = 8;                                   // vocabulary entries per thread per strip
 constexpr int kStrip = kWalkThreads * kEpt;               // 4096
 constexpr int kMaxStrips = 64;                            // V <= 262144
@@ -60,6 +65,45 @@ __device__ __forceinline__ void load8(const T* __restrict__ row, int i0, int V, 
 // ---------------------------------------------------------------------------------------------
 // K3: row statistics
 // ---------------------------------------------------------------------------------------------
+// Eight bf16 logits (one 16-byte vector starting at index ib) folded into a thread's running
+// statistics: maximum m, sum s of exp2((x - m) * k2), lowest index arg of the largest value bestv,
+// non-finite flag.  Maximum and minimum are taken on packed bf16 pairs with NaN propagation, so one
+// comparison of each against the finite range finds NaN and both infinities.
+__device__ __forceinline__ void stats8_bf16(const uint4& v, int ib, float k2, float& m, float& s, float& bestv, int& arg,
+                                            int& flag)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    __nv_bfloat162 h[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) h[j] = *reinterpret_cast<const __nv_bfloat162*>(&w[j]);
+    const __nv_bfloat162 mx2 = __hmax2_nan(__hmax2_nan(h[0], h[1]), __hmax2_nan(h[2], h[3]));
+    const __nv_bfloat162 mn2 = __hmin2_nan(__hmin2_nan(h[0], h[1]), __hmin2_nan(h[2], h[3]));
+    const float hi0 = __low2float(mx2), hi1 = __high2float(mx2), lo0 = __low2float(mn2), lo1 = __high2float(mn2);
+    if (!(hi0 <= 3.0e38f && hi1 <= 3.0e38f && lo0 >= -3.0e38f && lo1 >= -3.0e38f)) flag = 1;
+    const float cm = fmaxf(hi0, hi1);
+    if (cm > bestv) {                                    // rare after the first vectors: find the first element equal to it
+        bestv = cm;
+#pragma unroll
+        for (int j = 7; j >= 0; --j) {
+            const float x = __uint_as_float((j & 1) ? (w[j >> 1] & 0xffff0000u) : (w[j >> 1] << 16));
+            if (x == cm) arg = ib + j;
+        }
+    }
+    if (cm > m) { s *= ex2((m - cm) * k2); m = cm; }
+    const float nmk = -m * k2;
+    uint64_t acc = f2_pack(0.f, 0.f);
+    const uint64_t k22 = f2_pack(k2, k2), nmk2 = f2_pack(nmk, nmk);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float x0, x1;
+        f2_unpack(f2_fma(f2_pack(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xffff0000u)), k22, nmk2), x0, x1);
+        acc = f2_add(acc, f2_pack(ex2(x0), ex2(x1)));
+    }
+    float a0, a1;
+    f2_unpack(acc, a0, a1);
+    s += a0 + a1;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) row_stats_kernel(const T* __restrict__ tl, const T* __restrict__ dl, int V,
                                                         int n_rows, int nch, int chunk_elems, float k2,
@@ -77,6 +121,16 @@ __global__ void __launch_bounds__(256) row_stats_kernel(const T* __restrict__ tl
     for (int i0 = lo + tid * kEpt; i0 < hi; i0 += 256 * kEpt * 2) {
         float x[2][kEpt];
         const int i1 = i0 + 256 * kEpt;
+        if constexpr (sizeof(T) == 2) {
+            // bf16 rows, both 8-element vectors whole: packed path (about 4 instructions per logit)
+            if (vec_ok && i1 + kEpt <= hi) {
+                const uint4 v0 = *reinterpret_cast<const uint4*>(base + i0);
+                const uint4 v1 = *reinterpret_cast<const uint4*>(base + i1);
+                stats8_bf16(v0, i0, k2, m, s, bestv, arg, flag);
+                stats8_bf16(v1, i1, k2, m, s, bestv, arg, flag);
+                continue;
+            }
+        }
         load8(base, i0, hi, vec_ok, x[0]);
         if (i1 < hi) load8(base, i1, hi, vec_ok, x[1]);
 #pragma unroll
@@ -183,43 +237,54 @@ __device__ __forceinline__ float weight_at(float tx, float dx, int idx, int leve
     return fmaxf(p - q, 0.f);
 }
 
-// Sum of weight_at(., level) over the vocabulary, strip by strip, in double; fills sh.strip[].
+// Sum of weight_at(., level) over the vocabulary, strip by strip, in double; fills sh.strip[] of
+// every CTA of the cluster.  CTA `rank` computes strips rank, rank + kWalkCluster, ...
 template <typename T>
 __device__ double full_pass(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok, int level,
                             int mode, WalkShared& sh, float k2)
 {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x, n_strips = (V + kStrip - 1) / kStrip;
-    for (int s0 = 0; s0 < n_strips; s0 += 2) {
+    for (int sa = rank; sa < n_strips; sa += 2 * kWalkCluster) {
         float tx[2][kEpt], dx[2][kEpt];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-            const int i0 = (s0 + u) * kStrip + tid * kEpt;
-            if (s0 + u < n_strips) {
+            const int st = sa + u * kWalkCluster;
+            const int i0 = st * kStrip + tid * kEpt;
+            if (st < n_strips) {
                 load8(trow, i0, V, vec_ok, tx[u]);
                 if (level > 0) load8(drow, i0, V, vec_ok, dx[u]);
             }
         }
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-            if (s0 + u >= n_strips) break;
-            const int i0 = (s0 + u) * kStrip + tid * kEpt;
+            const int st = sa + u * kWalkCluster;
+            if (st >= n_strips) break;
+            const int i0 = st * kStrip + tid * kEpt;
             double acc = 0.0;
 #pragma unroll
             for (int j = 0; j < kEpt; ++j)
                 acc += (double)weight_at(tx[u][j], level > 0 ? dx[u][j] : 0.f, i0 + j, level, mode, sh, k2);
             acc = warp_sum(acc);
-            if ((tid & 31) == 0) sh.warp_part[s0 + u][tid >> 5] = acc;
+            if ((tid & 31) == 0) sh.warp_part[st][tid >> 5] = acc;
         }
     }
     __syncthreads();
-    if (tid < n_strips) {
-        double a = 0.0;
-        for (int w = 0; w < kWalkThreads / 32; ++w) a += sh.warp_part[tid][w];
-        sh.strip[tid] = a;
+    // every CTA has finished reading the strip sums of the previous pass: they may be overwritten
+    cluster.sync();
+    for (int i = tid; i < kMaxStrips * kWalkCluster; i += kWalkThreads) {
+        const int st = i / kWalkCluster, peer = i % kWalkCluster;
+        if (st < n_strips && st % kWalkCluster == rank) {
+            double a = 0.0;
+            for (int w = 0; w < kWalkThreads / 32; ++w) a += sh.warp_part[st][w];
+            *cluster.map_shared_rank(&sh.strip[st], peer) = a;
+        }
     }
-    __syncthreads();
+    cluster.sync();
     double tot = 0.0;
-    for (int s = 0; s < n_strips; ++s) tot += sh.strip[s];
+    for (int st = 0; st < n_strips; ++st) tot += sh.strip[st];
     return tot;
 }
 
@@ -297,7 +362,8 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     WalkShared& sh = *reinterpret_cast<WalkShared*>(smem_raw);
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int b = blockIdx.x / kWalkCluster, tid = threadIdx.x;
+    const bool writer = blockIdx.x % kWalkCluster == 0;            // the CTA of the cluster that writes the outputs
     const int32_t* par = parent + (size_t)b * Tn;
     const int32_t* tok = tokens + (size_t)b * Tn;
     const int32_t* own = con_owner ? con_owner + (size_t)b * C : nullptr;
@@ -333,8 +399,8 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
     __syncthreads();
     int32_t* pth = path + (size_t)b * kPathLen;
     if (sh.code != INT_MAX) {
-        if (tid < kPathLen) pth[tid] = tid == 0 ? 0 : -1;
-        if (tid == 0) {
+        if (writer && tid < kPathLen) pth[tid] = tid == 0 ? 0 : -1;
+        if (writer && tid == 0) {
             accept_len[b] = 0; next_token[b] = -1;
             if (future_row) future_row[b] = -1;
             if (counters) { counters[4 * b] = 0; counters[4 * b + 1] = 0; counters[4 * b + 2] = 0; counters[4 * b + 3] = 0; }
@@ -371,7 +437,7 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
             sh.len = depth[best];
             for (int a = best, k = sh.len; a >= 0; a = par[a], --k) sh.path[k] = a;
             sh.cur = best;
-            next_token[b] = sh.amax[best];
+            if (writer) next_token[b] = sh.amax[best];
         }
         __syncthreads();
     } else {
@@ -447,24 +513,24 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
             if (sh.done == 2) { final_level = 0; have_strips = false; }
             if (!have_strips) full_pass(trow, drow, V, vec_ok, final_level, mode, sh, k2);
             const int pick = locate(trow, drow, V, vec_ok, final_level, mode, sh, k2, u0);
-            if (tid == 0) next_token[b] = pick;
+            if (writer && tid == 0) next_token[b] = pick;
             break;
         }
         __syncthreads();
         if (sh.done == 3) {              // path buffer exhausted
-            if (tid < kPathLen) pth[tid] = tid == 0 ? 0 : -1;
-            if (tid == 0) {
+            if (writer && tid < kPathLen) pth[tid] = tid == 0 ? 0 : -1;
+            if (writer && tid == 0) {
                 accept_len[b] = 0; next_token[b] = -1;
                 if (future_row) future_row[b] = -1;
                 if (status) status[b] = CONFU_ST_TOO_DEEP;
             }
             return;
         }
-        if (sh.done == 2 && tid == 0 && status) status[b] = CONFU_ST_DEGENERATE;
+        if (sh.done == 2 && writer && tid == 0 && status) status[b] = CONFU_ST_DEGENERATE;
     }
     // ---- outputs ----
-    if (tid < kPathLen) pth[tid] = tid <= sh.len ? sh.path[tid] : -1;
-    if (tid == 0) {
+    if (writer && tid < kPathLen) pth[tid] = tid <= sh.len ? sh.path[tid] : -1;
+    if (writer && tid == 0) {
         accept_len[b] = sh.len;
         if (future_row) {
             int fr = -1;
@@ -511,10 +577,21 @@ static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, 
         if (e != cudaSuccess) return e;
         attr_done[ti] = true;
     }
-    accept_walk_kernel<T><<<B, kWalkThreads, smem, st>>>(Tn, C, V, (const T*)tl, (const T*)dl, tokens, parent,
-                                                         con_owner, uniforms, temperature, mode, nch, n_rows, stats,
-                                                         accept_len, path, next_token, future_row, counters, status);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)B * kWalkCluster);
+    cfg.blockDim = dim3(kWalkThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kWalkCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, accept_walk_kernel<T>, Tn, C, V, (const T*)tl, (const T*)dl, tokens, parent, con_owner,
+                              uniforms, temperature, mode, nch, n_rows, stats, accept_len, path, next_token, future_row,
+                              counters, status);
 }
 
 cudaError_t launch_accept(const Ctx*, int B, int T, int C, int V, int logit_dtype, const void* tl, const void* dl,
