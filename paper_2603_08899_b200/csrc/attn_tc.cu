@@ -1,29 +1,22 @@
 // Tensor-core tree attention for sm_100a: TMA-staged bf16 K/V tiles, tcgen05.mma with TMEM
 // accumulators, warp-specialised online softmax, stream-K split over the ragged batch.
 //
-// Work: the flat list of 128-key tiles of all (sequence, kv head) pairs is cut into contiguous
-// shares on a cost line (see the plan).  For a pair the query block is the R rows x G heads that
-// share the kv head: two M tiles of 128 rows (32 rows x G heads each, padded when G < 4).  A share
-// is walked by a UNIT of two CTAs, one per M tile; both stream the same K/V tiles at the same
-// time, so HBM delivers each tile once and the second reader finds it in L2.  (R <= 32: one M tile,
-// a unit is one CTA.)  Per CTA and key tile g:
-//     S_g = Q K_g^T           tcgen05.mma, A and B from shared memory (K-major, 128B swizzle),
-//                             into TMEM buffer S[g & 1]
-//     P_g = exp2(S_g*c - m)   one thread per row: tcgen05.ld, mask (last tiles only), tcgen05.st as bf16
-//                             into TMEM buffer P[g & 1]
-//     O  += P_g V_g           tcgen05.mma, A from TMEM, B = V tile in shared memory (MN-major)
-// S and P have two buffers each and do not overlay, so Q K^T of tile g+1 is issued before P_g
-// exists: the tensor pipe and the exponentials (MUFU) overlap instead of alternating.  The two
-// softmax warpgroups take alternate key tiles; both feed the same accumulator O, so they share one
-// reference maximum per row (shared memory), decided tile by tile in order; a warpgroup rescales
-// its own running sum lazily when it finds the maximum moved, and the rare move itself (past 2^8)
-// rescales O after the tensor pipe has drained the previous tile.
-// The tensor pipe holds about one instruction ahead of the issuing thread, so that thread does as
-// little as possible between MMAs: K/V travel in stages of [V of key tile g-1 | K of key tile g]
-// with one full and one empty barrier each.  Prefix tiles need no mask; the ancestor bitmask (one
-// 64-bit word per row, in a register) is applied only to the tiles that hold the tree slots, the
-// ragged tail and the soft-prompt entries.  A share that does not cover a whole pair writes an
-// unnormalised partial (O, m, l) that combine_kernel merges in a fixed order.
+// One persistent CTA per SM walks a contiguous range of the flat list of 128-key tiles of all
+// (sequence, kv head) pairs.  For a pair the query block is the R rows x G heads that share the kv
+// head: two M tiles of 128 rows (32 rows x G heads each, padded when G < 4).  Per key tile:
+//     S_t = Q_t K^T           tcgen05.mma, A and B from shared memory (K-major, 128B swizzle)
+//     P_t = exp2(S_t*c - m)   one thread per row: tcgen05.ld, mask (last tiles only), tcgen05.st as bf16
+//                             over the S columns
+//     O_t += P_t V            tcgen05.mma, A from TMEM, B = V tile in shared memory (MN-major)
+// Each M tile has its own softmax warpgroup; the two run out of phase, so that while one computes
+// exponentials the tensor pipe serves the other (P V, then the next Q K^T).  The tensor pipe holds
+// about one instruction ahead of the issuing thread, so whatever that thread does between MMAs is
+// idle pipe time: K/V travel in stages of [V of key tile g-1 | K of key tile g] with one full and
+// one empty barrier each, which leaves the issuing thread three waits and three commits per key
+// tile.  Prefix tiles need no mask; the ancestor bitmask (one 64-bit word per row, in a register) is applied only to
+// the tiles that hold the tree slots, the ragged tail and the soft-prompt entries.  A range that
+// does not cover a whole pair writes an unnormalised partial (O, m, l) that combine_kernel merges
+// in a fixed order.
 //
 // Every wait on an mbarrier is bounded (wall-clock limit); on expiry the CTA raises an abort flag,
 // every role leaves its loop, tensor memory is released and CONFU_ST_TIMEOUT is reported.
@@ -36,29 +29,22 @@ namespace confu {
 
 namespace tc {
 
-constexpr int kThreads = 384;            // warps 0-3: softmax of even key tiles, 4-7: of odd key tiles, 8: TMA of Q and K, 9: Q K^T, 10: P V, 11: TMA of V
-constexpr int kStages = 3;               // slots of the K ring and of the V ring (key tile g uses slot g % kStages of each)
+constexpr int kThreads = 384;            // warps 0-3: softmax of M tile 0, 4-7: of M tile 1, 8: TMA, 9: MMA
+constexpr int kStages = 2;               // ring of stages; stage g = [V of the CTA's g-1st key tile | K of its g-th]
 constexpr int kD = 128;
 constexpr int kTileBytes = kTileKeys * kD * 2;      // 32 KB
 constexpr int kHalfTile = kTileBytes / 2;           // one 64-wide half of the head dim: [128 rows][128 B]
-constexpr int kQBytes = kTileBytes;                 // the CTA's M tile
-constexpr uint32_t kTmemCols = 512;                 // O | S0 | S1 (128 columns each) | P0 | P1 (64 each)
-constexpr uint32_t kColO = 0, kColS = 128, kColP = 384;
+constexpr int kQBytes = 2 * kTileBytes;             // two M tiles
+constexpr uint32_t kTmemCols = 512;                 // S0 | S1 | O0 | O1, 128 columns each; P_t overlays S_t
 constexpr float kRescaleThreshold = 8.f;            // lazy rescale: move the reference max only past 2^8
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct SharedStorage {
     alignas(1024) uint8_t q[kQBytes];
-    alignas(1024) uint8_t k[kStages][kTileBytes];
-    alignas(1024) uint8_t v[kStages][kTileBytes];
+    alignas(1024) uint8_t kv[kStages][2][kTileBytes];    // [stage][0: V tile, 1: K tile]
     alignas(8) uint64_t q_full, q_empty;
-    uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-    uint64_t s_full[2], s_free[2], p_full[2];   // per S / P buffer (key tile parity); s_free: S read into registers
-    uint64_t o_done, o_free;            // last P V of a pair / range complete; O read out by both warpgroups
-    uint64_t turn[2];                   // turn[w]: warpgroup w may decide the reference maximum of its next tile
-    uint64_t seg_sync[2];               // both warpgroups have finished the tiles of a pair / range; have published their sums
-    float m_sh[2][128];                 // [range parity][row]: reference maximum (log2 domain)
-    float l_part[2][128];               // [warpgroup][row]: the warpgroup's sum under the final reference maximum
+    uint64_t kv_full[kStages], kv_empty[kStages];
+    uint64_t s_full[2], p_full[2], o_done[2];
     uint32_t tmem_base;
     int abort;
 };
@@ -72,7 +58,7 @@ struct Params {
     __nv_bfloat16* out;
     float* lse;
     int32_t* status;
-    int n_mt;            // M tiles in use (R > 32 ? 2 : 1) = CTAs per unit
+    int n_mt;            // M tiles in use (R > 32 ? 2 : 1)
     int G;
     float c;             // sm_scale * log2(e)
 };
@@ -98,21 +84,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// One non-blocking look at a barrier.  The issuing thread takes it well before it needs the answer
-// (a branch on a freshly loaded value costs it ~150 cycles of idle tensor pipe, one on an old
-// value next to nothing) and falls back to mbar_wait when the answer was "not yet".
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
@@ -236,14 +207,13 @@ struct Segment {
 
 struct Walker {
     const PlanView pv;
-    int64_t f, f1;             // this unit's share of the cost line: positions [f, f1)
+    int64_t f, f1;             // this CTA's share of the cost line: positions [f, f1)
     int cta;
     const Params& prm;
-    // cta_: index of the unit (the CTAs of a unit walk the same share)
     __device__ Walker(const PlanView& v, const Params& p, int cta_) : pv(v), cta(cta_), prm(p)
     {
         const int64_t N = v.hdr->n_tiles;
-        const int64_t n = v.hdr->n_units;
+        const int64_t n = v.hdr->n_ctas;
         f = (int64_t)cta_ * N / n;
         f1 = (int64_t)(cta_ + 1) * N / n;
     }
@@ -283,125 +253,144 @@ struct Walker {
 };
 
 // ------------------------------------------------------------------------------------ roles
-// Key tiles of the unit's share, all pairs together, are numbered g = 0..n-1 in walking order; K
-// and V tiles travel in rings of their own, because Q K^T runs up to two tiles ahead of P V.
-// Two producer threads, because the K ring is drained by the Q K^T thread and the V ring by the
-// P V thread two tiles later: a single producer waiting for a V slot would hold back the K tiles.
-__device__ void k_producer_role(SharedStorage& sh, const Params& prm, const PlanView& pv, int unit, int mt,
-                                const CUtensorMap* q_map, const CUtensorMap* k_map, const CUtensorMap* ks_map)
+// Key tiles of the CTA's share, all pairs together, are numbered g = 0..n-1 in walking order; stage
+// g of the ring carries V of tile g-1 and K of tile g (stage 0 has no V, stage n no K).
+__device__ int count_tiles(const Params& prm, const PlanView& pv)
 {
-    Walker w(pv, prm, unit);
+    Walker w(pv, prm, blockIdx.x);
     Segment s;
-    uint32_t g = 0, seg = 0;           // running tile / range counters
+    int n = 0;
+    while (w.next(s)) n += s.t1 - s.t0;
+    return n;
+}
+
+struct TileRef {                       // where a key tile's K and V come from
+    int g, z;                          // kv head, first slot (row) of the tile
+    bool soft;                         // the soft-prompt tile
+};
+
+__device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanView& pv, const CUtensorMap* q_map,
+                              const CUtensorMap* k_map, const CUtensorMap* v_map, const CUtensorMap* ks_map,
+                              const CUtensorMap* vs_map)
+{
+    const int n_total = count_tiles(prm, pv);
+    Walker w(pv, prm, blockIdx.x);
+    Segment s;
+    uint32_t stage = 0, seg = 0;       // running stage / pair counters
     const int R = prm.d.T + prm.d.C;
     const uint32_t q_box_bytes = 32u * prm.G * 128u;
+    TileRef prev = {0, 0, false};
+    bool have_prev = false;
+    // fills stage `stage` with V of `prev` (if any) and K of `cur` (if any)
+    auto fill = [&](const TileRef* cur) -> bool {
+        const uint32_t st = stage % kStages;
+        if (!mbar_wait(&sh.kv_empty[st], ((stage / kStages) & 1) ^ 1, &sh.abort)) return false;
+        mbar_arrive_expect_tx(&sh.kv_full[st], (have_prev ? kTileBytes : 0) + (cur ? kTileBytes : 0));
+        if (have_prev) {
+            const CUtensorMap* m = prev.soft ? vs_map : v_map;
+            tma_load_3d(sh.kv[st][0], m, &sh.kv_full[st], 0, prev.g, prev.z);
+            tma_load_3d(sh.kv[st][0] + kHalfTile, m, &sh.kv_full[st], 64, prev.g, prev.z);
+        }
+        if (cur) {
+            const CUtensorMap* m = cur->soft ? ks_map : k_map;
+            tma_load_3d(sh.kv[st][1], m, &sh.kv_full[st], 0, cur->g, cur->z);
+            tma_load_3d(sh.kv[st][1] + kHalfTile, m, &sh.kv_full[st], 64, cur->g, cur->z);
+        }
+        ++stage;
+        return true;
+    };
     while (w.next(s)) {
-        for (int t = s.t0; t < s.t1; ++t, ++g) {
-            const bool soft = t >= s.nkt;                                // the soft-prompt tile
-            const int z = soft ? 0 : (int)(s.slot0 + (int64_t)t * kTileKeys);
-            const uint32_t st = g % kStages;
-            if (!mbar_wait(&sh.k_empty[st], ((g / kStages) & 1) ^ 1, &sh.abort)) return;
-            mbar_arrive_expect_tx(&sh.k_full[st], kTileBytes);
-            const CUtensorMap* km = soft ? ks_map : k_map;
-            tma_load_3d(sh.k[st], km, &sh.k_full[st], 0, s.g, z);
-            tma_load_3d(sh.k[st] + kHalfTile, km, &sh.k_full[st], 64, s.g, z);
+        for (int t = s.t0; t < s.t1; ++t) {
+            TileRef cur;
+            cur.g = s.g;
+            cur.soft = t >= s.nkt;
+            cur.z = cur.soft ? 0 : (int)(s.slot0 + (int64_t)t * kTileKeys);
+            // the stage first (it carries the previous pair's last V tile, which must not wait for
+            // the Q buffer), then, at the start of a pair, its Q (both M tiles, two 64-wide halves each)
+            if (!fill(&cur)) return;
             if (t == s.t0) {
-                // the CTA's Q tile of this pair (two 64-wide halves)
                 if (!mbar_wait(&sh.q_empty, (seg & 1) ^ 1, &sh.abort)) return;
-                mbar_arrive_expect_tx(&sh.q_full, 2u * q_box_bytes);
-                for (int kb = 0; kb < 2; ++kb)
-                    tma_load_3d(sh.q + kb * kHalfTile, q_map, &sh.q_full, kb * 64, s.g * prm.G, s.b * R + 32 * mt);
+                mbar_arrive_expect_tx(&sh.q_full, 2u * prm.n_mt * q_box_bytes);
+                for (int mt = 0; mt < prm.n_mt; ++mt)
+                    for (int kb = 0; kb < 2; ++kb)
+                        tma_load_3d(sh.q + (mt * 2 + kb) * kHalfTile, q_map, &sh.q_full, kb * 64, s.g * prm.G, s.b * R + 32 * mt);
             }
+            prev = cur;
+            have_prev = true;
         }
         ++seg;
     }
+    if (n_total > 0 && !fill(nullptr)) return;
 }
 
-__device__ void v_producer_role(SharedStorage& sh, const Params& prm, const PlanView& pv, int unit,
-                                const CUtensorMap* v_map, const CUtensorMap* vs_map)
+// One thread issues all tensor-core work.  Per stage g: P V of key tile g-1 for both M tiles (each
+// as soon as its P is there), Q K^T of key tile g for both, then the stage is released.
+template <bool kTwo>
+__device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem)
 {
-    Walker w(pv, prm, unit);
+    constexpr int kMt = kTwo ? 2 : 1;
+    Walker w(pv, prm, blockIdx.x);
     Segment s;
-    uint32_t g = 0;
-    while (w.next(s)) {
-        for (int t = s.t0; t < s.t1; ++t, ++g) {
-            const bool soft = t >= s.nkt;
-            const int z = soft ? 0 : (int)(s.slot0 + (int64_t)t * kTileKeys);
-            const uint32_t st = g % kStages;
-            if (!mbar_wait(&sh.v_empty[st], ((g / kStages) & 1) ^ 1, &sh.abort)) return;
-            mbar_arrive_expect_tx(&sh.v_full[st], kTileBytes);
-            const CUtensorMap* vm = soft ? vs_map : v_map;
-            tma_load_3d(sh.v[st], vm, &sh.v_full[st], 0, s.g, z);
-            tma_load_3d(sh.v[st] + kHalfTile, vm, &sh.v_full[st], 64, s.g, z);
+    uint32_t stage = 0, seg = 0;
+    // descriptor low words: Q tiles (K-major); a stage's K tile (K-major) and V tile (MN-major, its
+    // two 64-column halves kHalfTile apart) = stage 0's words + stage * stage size
+    const uint32_t q_lo = desc_lo(smem_u32(sh.q), 16);
+    const uint32_t v_lo0 = desc_lo(smem_u32(sh.kv[0][0]), kHalfTile), k_lo0 = desc_lo(smem_u32(sh.kv[0][1]), 16);
+    constexpr uint32_t kTileStep = kTileBytes >> 4, kStageStep = 2 * kTileStep;
+
+    // S_t = Q_t K^T: 8 steps of 16 head dims; step i sits in 64-column half i/4 at byte 32*(i%4) of the swizzled row
+    auto issue_qk = [&](int t, uint32_t kl) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t off = ((uint32_t)(i >> 2) * kHalfTile + (uint32_t)(i & 3) * 32u) >> 4;
+            mma_ss(tmem + t * 128, q_lo + t * kTileStep + off, kl + off, kIdescQK, i > 0 ? 1u : 0u);
         }
-    }
-}
+        tc_commit(&sh.s_full[t]);
+    };
+    // O_t += P_t V: 8 steps of 16 keys (2048 B of the V tile and 8 TMEM columns of bf16 pairs each);
+    // P sits in the first 64 columns of the S_t block
+    auto issue_pv = [&](int t, uint32_t vl, bool first_of_segment) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            mma_ts(tmem + 256 + t * 128, tmem + t * 128 + i * 8, vl + i * (2048u >> 4), kIdescPV,
+                   (first_of_segment && i == 0) ? 0u : 1u);
+    };
+    // one stage: P V of the previous key tile (if any), Q K^T of the current one (if any)
+    bool have_prev = false, prev_first = false, prev_last = false;
+    auto run_stage = [&](bool have_cur, bool cur_first, bool cur_last) -> bool {
+        const uint32_t st = stage % kStages;
+        if (!mbar_wait(&sh.kv_full[st], (stage / kStages) & 1, &sh.abort)) return false;
+        if (have_cur && cur_first && !mbar_wait(&sh.q_full, seg & 1, &sh.abort)) return false;
+        tc_fence_after();
+        const uint32_t vl = v_lo0 + st * kStageStep, kl = k_lo0 + st * kStageStep;
+#pragma unroll
+        for (int t = 0; t < kMt; ++t) {
+            if (have_prev) {
+                // (At the start of a pair this P V overwrites the previous pair's O_t; the softmax
+                // threads hand P over only after they have read that O_t out.)
+                if (!mbar_wait(&sh.p_full[t], (stage - 1) & 1, &sh.abort)) return false;
+                tc_fence_after();
+                issue_pv(t, vl, prev_first);
+                if (prev_last) tc_commit(&sh.o_done[t]);
+            }
+            if (have_cur) issue_qk(t, kl);
+        }
+        tc_commit(&sh.kv_empty[st]);
+        if (have_cur && cur_last) tc_commit(&sh.q_empty);               // last Q K^T of the pair has been issued
+        ++stage;
+        have_prev = have_cur;
+        prev_first = cur_first;
+        prev_last = cur_last;
+        return true;
+    };
 
-// Two threads issue the tensor-core work, one per kind, so that the barrier traffic of one
-// overlaps the instruction issue of the other (the tensor pipe runs hardly ahead of its issuing
-// thread, but it interleaves two issuing threads without gaps).
-//
-// The Q K^T thread: key tile g into S[g & 1], free once the softmax threads have read tile g-2
-// out of it.  Q K^T thus runs up to two tiles ahead of P V, and a softmax warpgroup that hands P
-// over finds its next S waiting.
-__device__ void mma_qk_role(SharedStorage& sh, const Params& prm, const PlanView& pv, int unit, uint32_t tmem)
-{
-    Walker w(pv, prm, unit);
-    Segment s;
-    uint32_t g = 0, seg = 0;
-    // descriptor low words: the Q tile and slot 0 of the K ring (both K-major); slot i = slot 0's word + i * tile size
-    const uint32_t q_lo = desc_lo(smem_u32(sh.q), 16), k_lo0 = desc_lo(smem_u32(sh.k[0]), 16);
-    constexpr uint32_t kSlotStep = kTileBytes >> 4;
     while (w.next(s)) {
         const int n_tiles = s.t1 - s.t0;
-        for (int j = 0; j < n_tiles; ++j, ++g) {
-            const uint32_t st = g % kStages;
-            if (!mbar_wait(&sh.k_full[st], (g / kStages) & 1, &sh.abort)) return;
-            if (j == 0 && !mbar_wait(&sh.q_full, seg & 1, &sh.abort)) return;
-            if (g >= 2 && !mbar_wait(&sh.s_free[g & 1], ((g - 2) >> 1) & 1, &sh.abort)) return;
-            tc_fence_after();
-            // S = Q K^T: 8 steps of 16 head dims; step k sits in 64-column half k/4 at byte 32*(k%4) of the swizzled row
-            const uint32_t kl = k_lo0 + st * kSlotStep, s_tmem = tmem + kColS + (g & 1) * 128;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t off = ((uint32_t)(k >> 2) * kHalfTile + (uint32_t)(k & 3) * 32u) >> 4;
-                mma_ss(s_tmem, q_lo + off, kl + off, kIdescQK, k > 0 ? 1u : 0u);
-            }
-            tc_commit(&sh.s_full[g & 1]);
-            tc_commit(&sh.k_empty[st]);
-            if (j + 1 == n_tiles) tc_commit(&sh.q_empty);               // last Q K^T of the pair has been issued
-        }
+        for (int j = 0; j < n_tiles; ++j)
+            if (!run_stage(true, j == 0, j + 1 == n_tiles)) return;
         ++seg;
     }
-}
-
-// The P V thread: O += P V of key tile g as soon as its P is there.
-__device__ void mma_pv_role(SharedStorage& sh, const Params& prm, const PlanView& pv, int unit, uint32_t tmem)
-{
-    Walker w(pv, prm, unit);
-    Segment s;
-    uint32_t g = 0, seg = 0;
-    const uint32_t v_lo0 = desc_lo(smem_u32(sh.v[0]), kHalfTile);      // V tile, MN-major, halves kHalfTile apart
-    constexpr uint32_t kSlotStep = kTileBytes >> 4;
-    while (w.next(s)) {
-        const int n_tiles = s.t1 - s.t0;
-        for (int j = 0; j < n_tiles; ++j, ++g) {
-            const uint32_t st = g % kStages;
-            if (!mbar_wait(&sh.v_full[st], (g / kStages) & 1, &sh.abort)) return;
-            // the first P V of a pair overwrites O: both warpgroups must have read the previous pair's O out
-            if (j == 0 && seg > 0 && !mbar_wait(&sh.o_free, (seg - 1) & 1, &sh.abort)) return;
-            if (!mbar_wait(&sh.p_full[g & 1], (g >> 1) & 1, &sh.abort)) return;
-            tc_fence_after();
-            // O += P V: 8 steps of 16 keys (2048 B of the V tile and 8 TMEM columns of bf16 pairs each)
-            const uint32_t vl = v_lo0 + st * kSlotStep, p_tmem = tmem + kColP + (g & 1) * 64;
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-                mma_ts(tmem + kColO, p_tmem + k * 8, vl + k * (2048u >> 4), kIdescPV, (j == 0 && k == 0) ? 0u : 1u);
-            if (j + 1 == n_tiles) tc_commit(&sh.o_done);
-            tc_commit(&sh.v_empty[st]);                                  // fires when this tile's P V has completed
-        }
-        ++seg;
-    }
+    if (have_prev) run_stage(false, false, false);
 }
 
 // Which of the 128 keys of tile `t` may row r see.  lo: keys 0..63 of the tile, hi: 64..127.
@@ -442,188 +431,138 @@ __device__ __forceinline__ float max128(const uint32_t (&sv)[128])
     return fmaxf(fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3])), fmaxf(fmaxf(a[4], a[5]), fmaxf(a[6], a[7])));
 }
 
-// exp2(s*c - m) of 64 scores -> 32 packed bf16 pairs; returns their fp32 sum (four independent
-// partial sums, so that the additions do not form one long dependent chain)
+// exp2(s*c - m) of 64 scores -> 32 packed bf16 pairs; returns their fp32 sum
 __device__ __forceinline__ float weights64(const uint32_t* sv, float c, float neg_m, uint32_t (&pk)[32])
 {
-    uint64_t sum2[4] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f), f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
+    uint64_t sum2 = f2_pack(0.f, 0.f);
     const uint64_t c2 = f2_pack(c, c), nm2 = f2_pack(neg_m, neg_m);
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
         float x0, x1;
         f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1])), c2, nm2), x0, x1);
         const float p0 = ex2(x0), p1 = ex2(x1);
-        sum2[j & 3] = f2_add(sum2[j & 3], f2_pack(p0, p1));
+        sum2 = f2_add(sum2, f2_pack(p0, p1));
         pk[j] = pack_bf16(p0, p1);
     }
     float s0, s1;
-    f2_unpack(f2_add(f2_add(sum2[0], sum2[1]), f2_add(sum2[2], sum2[3])), s0, s1);
+    f2_unpack(sum2, s0, s1);
     return s0 + s1;
 }
 
-// running sum l held under reference m_from, re-expressed under m_to >= m_from
-__device__ __forceinline__ float rebase(float l, float m_from, float m_to)
-{
-    return (m_from == m_to) ? l : ((m_from == -INFINITY) ? 0.f : l * ex2(m_from - m_to));
-}
-
-// Softmax warpgroup wg (0: even key tiles of the CTA's stream, 1: odd), one thread per query row.
-__device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanView& pv, int unit, int mt, uint32_t tmem,
-                             int wg)
+__device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem, int t /*M tile*/)
 {
     const int lane_row = threadIdx.x & 127;                 // row of the M tile = TMEM lane
     const int warp_in_wg = (threadIdx.x >> 5) & 3;
     const uint32_t lane_base = (uint32_t)(warp_in_wg * 32) << 16;
-    const uint32_t s_addr = tmem + lane_base + kColS + wg * 128;
-    const uint32_t p_addr = tmem + lane_base + kColP + wg * 64;
-    const uint32_t o_addr = tmem + lane_base + kColO;
+    const uint32_t s_addr = tmem + lane_base + t * 128;
+    const uint32_t o_addr = tmem + lane_base + 256 + t * 128;
     const int G = prm.G, T = prm.d.T, R = prm.d.T + prm.d.C, S = prm.d.S, Hq = prm.d.Hq;
-    const int r = 32 * mt + lane_row / G, hl = lane_row % G;
+    const int r = 32 * t + lane_row / G, hl = lane_row % G;
     const bool row_valid = lane_row < 32 * G && r < R;
     const float c = prm.c;
 
-    Walker w(pv, prm, unit);
+    Walker w(pv, prm, blockIdx.x);
     Segment s;
-    uint32_t g0 = 0;            // stream index of the current range's first tile
-    uint32_t k = 0;             // key tiles this warpgroup has taken so far (phase of its S / P buffer barriers)
-    uint32_t seg = 0;
+    uint32_t n_s = 0, seg = 0;
     while (w.next(s)) {
-        const int n_tiles = s.t1 - s.t0;
         const uint64_t mask = row_valid ? pv.mask[(size_t)s.b * kMaxRows + r] : 0ull;
-        float* m_row = &sh.m_sh[seg & 1][lane_row];
-        float m_loc = -INFINITY, l_loc = 0.f;          // this warpgroup's running sum and the reference it is held under
-        for (int j = (int)((wg - g0) & 1u); j < n_tiles; j += 2, ++k) {
-            const int tile = s.t0 + j;
-            const uint32_t g = g0 + j;
-            if (!mbar_wait(&sh.s_full[wg], k & 1, &sh.abort)) return;
+        float m_ref = -INFINITY, l = 0.f;
+        for (int tile = s.t0; tile < s.t1; ++tile) {
+            if (!mbar_wait(&sh.s_full[t], n_s & 1, &sh.abort)) return;
+            ++n_s;
             tc_fence_after();
             uint32_t sv[128];
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(s_addr + q4 * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[q4 * 32]));
             tc_wait_ld();
-            tc_fence_before();
-            mbar_arrive(&sh.s_free[wg]);                 // the tensor pipe may write tile g+2's scores into this buffer
             const bool masked = tile >= s.nkt || (int64_t)(tile + 1) * kTileKeys > s.P;
             if (masked) {
                 uint64_t lo, hi;
                 visible_bits(s, tile, R, T, S, r, row_valid, mask, lo, hi);
 #pragma unroll
-                for (int jj = 0; jj < 64; ++jj) {
-                    if (!((lo >> jj) & 1ull)) sv[jj] = 0xff800000u;            // -inf
-                    if (!((hi >> jj) & 1ull)) sv[64 + jj] = 0xff800000u;
+                for (int j = 0; j < 64; ++j) {
+                    if (!((lo >> j) & 1ull)) sv[j] = 0xff800000u;            // -inf
+                    if (!((hi >> j) & 1ull)) sv[64 + j] = 0xff800000u;
                 }
             }
-            const float mx = row_valid ? max128(sv) : -INFINITY;
-            // The reference maxima are decided in stream order: tile g after tile g-1 (other warpgroup).
-            if (g > 0 && !mbar_wait(&sh.turn[wg], (wg ? k : k - 1) & 1, &sh.abort)) return;
-            const bool first = j == 0;
-            float m_cur = first ? -INFINITY : *m_row;
-            l_loc = rebase(l_loc, m_loc, m_cur);
-            const float m_new = fmaxf(m_cur, mx * c);
-            if (first) {
-                m_cur = m_new;
-                *m_row = m_cur;
+            const float m_new = fmaxf(m_ref, max128(sv) * c);
+            if (tile == s.t0) {
+                m_ref = m_new;
             } else {
-                const bool move = m_new - m_cur > kRescaleThreshold;         // false when both are -inf (NaN)
+                const bool move = m_new - m_ref > kRescaleThreshold;         // false when both are -inf (NaN)
                 if (__any_sync(0xffffffffu, move)) {
-                    // O must hold exactly the tiles before g: the V slot of tile g-1 is released when its
-                    // P V has completed, and the P V of tile g cannot start before this thread's P.
-                    if (!mbar_wait(&sh.v_empty[(g - 1) % kStages], ((g - 1) / kStages) & 1, &sh.abort)) return;
-                    tc_fence_after();
-                    const float alpha = move ? ex2(m_cur - m_new) : 1.f;
+                    const float alpha = move ? ex2(m_ref - m_new) : 1.f;
+                    if (move) { m_ref = m_new; l *= alpha; }
+                    // S_full of this tile implies the previous PV of this M tile has completed
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
                         uint32_t ov[32];
                         tmem_ld32(o_addr + q4 * 32, ov);
                         tc_wait_ld();
 #pragma unroll
-                        for (int jj = 0; jj < 32; ++jj) ov[jj] = __float_as_uint(__uint_as_float(ov[jj]) * alpha);
+                        for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
                         tmem_st32(o_addr + q4 * 32, ov);
-                    }
-                    tc_wait_st();
-                    if (move) {
-                        l_loc *= alpha;
-                        m_cur = m_new;
-                        *m_row = m_cur;
                     }
                 }
             }
-            m_loc = m_cur;
-            const float neg_m = (m_cur == -INFINITY) ? 0.f : -m_cur;
-            // masked scores are -inf and get weight exactly 0
+            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            // P overlays the first 64 columns of S_t (all of S_t is in registers by now); masked
+            // scores are -inf and get weight exactly 0
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t pk[32];
-                l_loc += weights64(&sv[64 * half], c, neg_m, pk);
-                // P buffer g & 1 last held tile g-2: its P V must have completed (V slot released)
-                // before the buffer is overwritten; by now that wait is usually over
-                if (half == 0 && g >= 2 && !mbar_wait(&sh.v_empty[(g - 2) % kStages], ((g - 2) / kStages) & 1, &sh.abort)) return;
-                // The turn passes on only now, after this tile's exponentials: the other warpgroup,
-                // which has loaded and reduced its scores meanwhile, decides its reference maximum
-                // next and then has the MUFU to itself.  The two exponential phases alternate
-                // instead of halving each other's rate, and P reaches the tensor pipe sooner.
-                if (half == 1) mbar_arrive(&sh.turn[wg ^ 1]);
-                tmem_st32(p_addr + 32 * half, pk);
+                l += weights64(&sv[64 * half], c, neg_m, pk);
+                tmem_st32(s_addr + 32 * half, pk);
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(&sh.p_full[wg]);
+            mbar_arrive(&sh.p_full[t]);
         }
-        g0 += n_tiles;
-        // ---- end of this pair / range: merge the two warpgroups' sums, write the CTA's rows ----
-        mbar_arrive(&sh.seg_sync[0]);                                    // every reference maximum of the range is final
-        if (!mbar_wait(&sh.seg_sync[0], seg & 1, &sh.abort)) return;
-        const float m_fin = *m_row;
-        sh.l_part[wg][lane_row] = rebase(l_loc, m_loc, m_fin);
-        mbar_arrive(&sh.seg_sync[1]);
-        if (!mbar_wait(&sh.seg_sync[1], seg & 1, &sh.abort)) return;
-        const float l = sh.l_part[0][lane_row] + sh.l_part[1][lane_row];
-        if (!mbar_wait(&sh.o_done, seg & 1, &sh.abort)) return;
+        // ---- epilogue of this pair / range ----
+        if (!mbar_wait(&sh.o_done[t], seg & 1, &sh.abort)) return;
         tc_fence_after();
         const int h = s.g * G + hl;
-        // each warpgroup takes 64 of the 128 output columns
         if (s.part_slot < 0) {
             const float inv_l = 1.f / l;
-            __nv_bfloat16* orow = prm.out + (((size_t)s.b * R + r) * Hq + h) * kD + 64 * wg;
+            __nv_bfloat16* orow = prm.out + (((size_t)s.b * R + r) * Hq + h) * kD;
 #pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2) {
+            for (int q4 = 0; q4 < 4; ++q4) {
                 uint32_t ov[32];
-                tmem_ld32(o_addr + 64 * wg + q2 * 32, ov);
+                tmem_ld32(o_addr + q4 * 32, ov);
                 tc_wait_ld();
                 if (row_valid) {
 #pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
+                    for (int j = 0; j < 4; ++j) {
                         uint4 pkt;
-                        pkt.x = pack_bf16(__uint_as_float(ov[8 * jj + 0]) * inv_l, __uint_as_float(ov[8 * jj + 1]) * inv_l);
-                        pkt.y = pack_bf16(__uint_as_float(ov[8 * jj + 2]) * inv_l, __uint_as_float(ov[8 * jj + 3]) * inv_l);
-                        pkt.z = pack_bf16(__uint_as_float(ov[8 * jj + 4]) * inv_l, __uint_as_float(ov[8 * jj + 5]) * inv_l);
-                        pkt.w = pack_bf16(__uint_as_float(ov[8 * jj + 6]) * inv_l, __uint_as_float(ov[8 * jj + 7]) * inv_l);
-                        *reinterpret_cast<uint4*>(orow + q2 * 32 + jj * 8) = pkt;
+                        pkt.x = pack_bf16(__uint_as_float(ov[8 * j + 0]) * inv_l, __uint_as_float(ov[8 * j + 1]) * inv_l);
+                        pkt.y = pack_bf16(__uint_as_float(ov[8 * j + 2]) * inv_l, __uint_as_float(ov[8 * j + 3]) * inv_l);
+                        pkt.z = pack_bf16(__uint_as_float(ov[8 * j + 4]) * inv_l, __uint_as_float(ov[8 * j + 5]) * inv_l);
+                        pkt.w = pack_bf16(__uint_as_float(ov[8 * j + 6]) * inv_l, __uint_as_float(ov[8 * j + 7]) * inv_l);
+                        *reinterpret_cast<uint4*>(orow + q4 * 32 + j * 8) = pkt;
                     }
                 }
             }
-            if (row_valid && wg == 0 && prm.lse)
-                prm.lse[((size_t)s.b * R + r) * Hq + h] = (m_fin + log2f(l)) * 0.6931471805599453f;
+            if (row_valid && prm.lse)
+                prm.lse[((size_t)s.b * R + r) * Hq + h] = (m_ref + log2f(l)) * 0.6931471805599453f;
         } else {
             float* slot = prm.partials + (size_t)s.part_slot * (partial_slot_bytes() / sizeof(float));
-            float* prow = slot + (size_t)(mt * 128 + lane_row) * kPartD + 64 * wg;
+            float* prow = slot + (size_t)(t * 128 + lane_row) * kPartD;
 #pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2) {
+            for (int q4 = 0; q4 < 4; ++q4) {
                 uint32_t ov[32];
-                tmem_ld32(o_addr + 64 * wg + q2 * 32, ov);
+                tmem_ld32(o_addr + q4 * 32, ov);
                 tc_wait_ld();
 #pragma unroll
-                for (int jj = 0; jj < 8; ++jj)
-                    *reinterpret_cast<uint4*>(prow + q2 * 32 + jj * 4) = make_uint4(ov[4 * jj], ov[4 * jj + 1], ov[4 * jj + 2], ov[4 * jj + 3]);
+                for (int j = 0; j < 8; ++j)
+                    *reinterpret_cast<uint4*>(prow + q4 * 32 + j * 4) = make_uint4(ov[4 * j], ov[4 * j + 1], ov[4 * j + 2], ov[4 * j + 3]);
             }
-            if (wg == 0) {
-                float* ml = slot + (size_t)kPartRows * kPartD;
-                ml[mt * 128 + lane_row] = m_fin;
-                ml[kPartRows + mt * 128 + lane_row] = l;
-            }
+            float* ml = slot + (size_t)kPartRows * kPartD;
+            ml[t * 128 + lane_row] = m_ref;
+            ml[kPartRows + t * 128 + lane_row] = l;
         }
+        // the P of the next range's first tile is only handed over after this point, which is what
+        // keeps the tensor pipe from overwriting O_t before it has been read
         tc_fence_before();
-        mbar_arrive(&sh.o_free);
         ++seg;
     }
 }
@@ -633,39 +572,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                     const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap ks_map,
                     const __grid_constant__ CUtensorMap vs_map, const Params prm)
 {
-    // The dynamic shared memory window starts at offset 0 of the CTA's shared memory (the kernel has
-    // no static shared memory), which is what gives the tiles their 1024-byte alignment; there is no
-    // room for alignment slack.  Checked below, reported as CONFU_ST_TIMEOUT's sibling: nothing runs.
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    SharedStorage& sh = *reinterpret_cast<SharedStorage*>(smem_raw);
-    if ((smem_u32(smem_raw) & 1023u) != 0) {
-        if (threadIdx.x == 0 && prm.status)
-            for (int b = 0; b < prm.d.B; ++b) prm.status[b] = CONFU_ST_TIMEOUT;
-        return;
-    }
+    extern __shared__ uint8_t smem_raw[];
+    SharedStorage& sh = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
-    // a unit = the n_mt CTAs (consecutive block indices) that walk one share, one per M tile
-    const int unit = (int)blockIdx.x / prm.n_mt, mt = (int)blockIdx.x % prm.n_mt;
-    if (unit >= pv.hdr->n_units) return;
+    if ((int)blockIdx.x >= pv.hdr->n_ctas) return;
     const int warp = threadIdx.x >> 5;
 
     if (threadIdx.x == 0) {
         mbar_init(&sh.q_full, 1);
         mbar_init(&sh.q_empty, 1);
-        for (int i = 0; i < kStages; ++i) {
-            mbar_init(&sh.k_full[i], 1); mbar_init(&sh.k_empty[i], 1);
-            mbar_init(&sh.v_full[i], 1); mbar_init(&sh.v_empty[i], 1);
-        }
+        for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
         for (int t = 0; t < 2; ++t) {
             mbar_init(&sh.s_full[t], 1);
-            mbar_init(&sh.s_free[t], 128);
             mbar_init(&sh.p_full[t], 128);
-            mbar_init(&sh.turn[t], 128);
+            mbar_init(&sh.o_done[t], 1);
         }
-        mbar_init(&sh.o_done, 1);
-        mbar_init(&sh.o_free, 256);
-        mbar_init(&sh.seg_sync[0], 256);
-        mbar_init(&sh.seg_sync[1], 256);
         sh.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -683,17 +604,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 
     if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
-        softmax_role(sh, prm, pv, unit, mt, tmem, warp >> 2);
+        const int t = warp >> 2;
+        if (t < prm.n_mt) softmax_role(sh, prm, pv, tmem, t);
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
         if (warp == 8) {
-            if ((threadIdx.x & 31) == 0) k_producer_role(sh, prm, pv, unit, mt, &q_map, &k_map, &ks_map);
-        } else if (warp == 11) {
-            if ((threadIdx.x & 31) == 0) v_producer_role(sh, prm, pv, unit, &v_map, &vs_map);
+            if ((threadIdx.x & 31) == 0) producer_role(sh, prm, pv, &q_map, &k_map, &v_map, &ks_map, &vs_map);
         } else if (warp == 9) {
-            if ((threadIdx.x & 31) == 0) mma_qk_role(sh, prm, pv, unit, tmem);
-        } else if (warp == 10) {
-            if ((threadIdx.x & 31) == 0) mma_pv_role(sh, prm, pv, unit, tmem);
+            if ((threadIdx.x & 31) == 0) {
+                if (prm.n_mt > 1) mma_role<true>(sh, prm, pv, tmem);
+                else mma_role<false>(sh, prm, pv, tmem);
+            }
         }
         __syncwarp();
     }
@@ -724,11 +645,11 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
     const int b = pair / prm.d.Hkv, g = pair % prm.d.Hkv;
     const int nt = pv.tiles[b];
     if (nt == 0 || t >= prm.n_mt) return;
-    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_units;
-    // key tile q of the pair sits at position F + q of the cost line; position x belongs to unit floor(((x + 1) * n - 1) / N)
+    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
+    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
     const int64_t F = pv.tile_base[b] + (int64_t)g * (nt + kPairOverheadTiles) + kPairOverheadTiles;
     const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
-    if (c_first == c_last) return;                      // one unit covered the pair and wrote the output itself
+    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
     const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t slot_floats = partial_slot_bytes() / sizeof(float);
@@ -830,16 +751,14 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     prm.n_mt = R > 32 ? 2 : 1;
     prm.G = G;
     prm.c = (d.sm_scale != 0.f ? d.sm_scale : 1.f / sqrtf((float)d.D)) * 1.4426950408889634f;
-    const size_t smem = sizeof(SharedStorage);
+    const size_t smem = sizeof(SharedStorage) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    // one CTA per (unit, M tile); the plan made at most sm_count / n_mt units
-    const int grid = ctx->sm_count / prm.n_mt * prm.n_mt;
-    attention_tc_kernel<<<grid, kThreads, smem, st>>>(q_map, k_map, v_map, ks_map, vs_map, prm);
+    attention_tc_kernel<<<ctx->sm_count, kThreads, smem, st>>>(q_map, k_map, v_map, ks_map, vs_map, prm);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     combine_kernel<<<dim3(d.B * d.Hkv, prm.n_mt), 256, 0, st>>>(prm);

@@ -23,15 +23,14 @@ constexpr int kTileKeys = 128;                  // keys per attention tile (tens
 //
 // The split-KV work is balanced on a "cost line": every (sequence, kv head) pair takes
 // tiles + kPairOverheadTiles consecutive positions (the overhead stands for loading Q, draining
-// the pipeline and writing the output once per pair), pairs in (sequence, head) order.  Unit c of n
+// the pipeline and writing the output once per pair), pairs in (sequence, head) order.  CTA c of n
 // gets positions [c*N/n, (c+1)*N/n); position q of a pair means key tile q - kPairOverheadTiles,
-// so a unit whose share ends inside a pair's overhead zone takes none of its tiles.
+// so a CTA whose share ends inside a pair's overhead zone takes none of its tiles.
 // ---------------------------------------------------------------------------
 constexpr int kPairOverheadTiles = 4;
 struct PlanHeader {
     int32_t B, Hkv, T, C, S, R;
-    int32_t n_units;           // shares of the cost line = units of the tensor-core attention launch
-                               // (a unit is one CTA per 128-row M tile of the query block: 2 when R > 32)
+    int32_t n_ctas;            // CTAs of the tensor-core attention launch (<= SM count)
     int32_t pad;
     int64_t n_tiles;           // length N of the cost line
 };

@@ -80,8 +80,7 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
         PlanHeader h;
         h.B = B; h.Hkv = d.Hkv; h.T = T; h.C = C; h.S = d.S; h.R = R;
         h.n_tiles = acc;
-        const int64_t max_units = R > 32 ? sm_count / 2 : sm_count;      // two CTAs (one per M tile) walk a share when R > 32
-        h.n_units = (int)(acc < max_units ? acc : max_units);
+        h.n_ctas = (int)(acc < (int64_t)sm_count ? acc : (int64_t)sm_count);
         h.pad = 0;
         *pv.hdr = h;
     }
