@@ -636,8 +636,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 }
 
 // Merge of the split-KV partials of one (sequence, kv head) pair, in CTA order (deterministic).
-// One block per (pair, M tile); a warp takes a row at a time, lane i the row's columns 4i..4i+3, so
-// partial rows are read and output rows written as whole 512- and 256-byte lines.
+// One block per (pair, M tile, 32 rows); a warp takes a row at a time (four rows in all), lane i the
+// row's columns 4i..4i+3, so partial rows are read and output rows written as whole 512- and
+// 256-byte lines.
 __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
 {
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
@@ -653,7 +654,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
     const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t slot_floats = partial_slot_bytes() / sizeof(float);
-    for (int lane_row = warp; lane_row < 32 * G; lane_row += 8) {
+    for (int lane_row = blockIdx.z * 32 + warp; lane_row < min(32 * G, (int)blockIdx.z * 32 + 32); lane_row += 8) {
         const int r = 32 * t + lane_row / G, hl = lane_row % G;
         if (r >= R) break;
         const int row = t * 128 + lane_row;
@@ -761,7 +762,7 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     attention_tc_kernel<<<ctx->sm_count, kThreads, smem, st>>>(q_map, k_map, v_map, ks_map, vs_map, prm);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    combine_kernel<<<dim3(d.B * d.Hkv, prm.n_mt), 256, 0, st>>>(prm);
+    combine_kernel<<<dim3(d.B * d.Hkv, prm.n_mt, 4), 256, 0, st>>>(prm);
     return cudaGetLastError();
 }
 
