@@ -29,8 +29,8 @@
  *     A sequence with a non-zero status has unspecified outputs.
  *
  * Row and slot conventions
- *   T tree rows (row 0 = root = the token emitted by the previous step), then C
- *   contemplate rows; R = T + C <= 64.  parent[b][0] = -1 and 0 <= parent[b][i] < i.
+ *   T <= 64 tree rows (row 0 = root = the token emitted by the previous step), then
+ *   C <= 64 contemplate rows; R = T + C <= 128.  parent[b][0] = -1 and 0 <= parent[b][i] < i.
  *   con_owner[b][k] in [0,T) is the tree node that contemplate row T+k sits behind.
  *   A layer's cache pool is [n_slots][Hkv][D]; sequence b owns slots
  *   seq_start[b] .. seq_start[b] + prefix_len[b] + R - 1: its prefix, then the K/V of
@@ -55,7 +55,7 @@ enum {
     CONFU_ERR_SHAPE = -2,        /* Hq % Hkv != 0, D not in {64,128}, T < 1, ... */
     CONFU_ERR_ALIGN = -3,        /* a device pointer is not 16-byte aligned */
     CONFU_ERR_WORKSPACE = -4,    /* workspace missing or too small */
-    CONFU_ERR_UNSUPPORTED = -5,  /* e.g. R > 64 */
+    CONFU_ERR_UNSUPPORTED = -5,  /* e.g. T > 64 or C > 64 */
     CONFU_ERR_CUDA = -6          /* a CUDA call failed: see confu_last_cuda_error */
 };
 
@@ -74,7 +74,8 @@ enum {
 
 enum { CONFU_BF16 = 0, CONFU_F32 = 1 };
 
-#define CONFU_MAX_ROWS  64      /* R = T + C */
+#define CONFU_MAX_TREE  64      /* T: tree rows (one 64-bit ancestor word per row) */
+#define CONFU_MAX_ROWS  128     /* R = T + C, with C <= 64: covers one contemplate row per node (R = 2T) */
 #define CONFU_MAX_DEPTH 63      /* path buffers hold CONFU_MAX_DEPTH + 1 node ids */
 
 typedef struct {
@@ -132,7 +133,8 @@ int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims,
  * denominators.  plan: a buffer filled by confu_tree_plan for these dims, lengths
  * and trees, or NULL to have the call build one in the workspace (then parent,
  * con_owner are read; otherwise they may be NULL).  Accumulation is fp32; bf16
- * inputs use the tensor-core path when D == 128 and Hq/Hkv <= 4.
+ * inputs use the tensor-core path when D == 128 and Hq/Hkv <= 4; it takes the
+ * query rows in groups of 64, so R > 64 streams the keys twice.
  * Needs the workspace.  All pointers device.
  */
 int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims,

@@ -12,7 +12,8 @@ import torch
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libconfu.so")
 
-MAX_ROWS = 64
+MAX_TREE = 64
+MAX_ROWS = 128
 MAX_DEPTH = 63
 BF16, F32 = 0, 1
 OK = 0

@@ -192,12 +192,12 @@ struct WalkShared {
     int code;
     int cur, len, k, nch, accepted, done, final_level;
     int path[kPathLen];
-    int ch[kMaxRows];
-    int xs[kMaxRows];          // rejected tokens at the current node
-    float invZ[kMaxRows];      // 1 / Z_j
-    float cs[kMaxRows];        // 1 / (1 - q_{j-1}(x_j))   (sibling_mode 1)
+    int ch[kMaxTree];
+    int xs[kMaxTree];          // rejected tokens at the current node
+    float invZ[kMaxTree];      // 1 / Z_j
+    float cs[kMaxTree];        // 1 / (1 - q_{j-1}(x_j))   (sibling_mode 1)
     float Mt, Md, invZt, invZd;
-    int amax[kMaxRows];
+    int amax[kMaxTree];
     double strip[kMaxStrips];
     double warp_part[kMaxStrips][kWalkThreads / 32];
     double scan[kWalkThreads / 32];
@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
         __syncthreads();
         if (tid == 0) {
             unsigned long long keep = 1ull;
-            int depth[kMaxRows];
+            int depth[kMaxTree];
             depth[0] = 0;
             int best = 0;
             for (int i = 1; i < Tn; ++i) {

@@ -18,7 +18,7 @@ int check_dims(const confu_dims* d)
     if (d->Hq % d->Hkv != 0) return CONFU_ERR_SHAPE;
     if (d->D != 64 && d->D != 128) return CONFU_ERR_SHAPE;
     if (d->kv_dtype != CONFU_BF16 && d->kv_dtype != CONFU_F32) return CONFU_ERR_ARG;
-    if (d->T + d->C > CONFU_MAX_ROWS) return CONFU_ERR_UNSUPPORTED;
+    if (d->T > CONFU_MAX_TREE || d->C > CONFU_MAX_TREE) return CONFU_ERR_UNSUPPORTED;
     if (!(d->sm_scale >= 0.f)) return CONFU_ERR_ARG;
     return CONFU_OK;
 }
@@ -194,7 +194,7 @@ int confu_tree_accept(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V
     if (logit_dtype != CONFU_BF16 && logit_dtype != CONFU_F32) return CONFU_ERR_ARG;
     if (sibling_mode != 0 && sibling_mode != 1) return CONFU_ERR_ARG;
     if (!(temperature >= 0.f)) return CONFU_ERR_ARG;
-    if (T > CONFU_MAX_ROWS || C > CONFU_MAX_ROWS || V > 262144) return CONFU_ERR_UNSUPPORTED;
+    if (T > CONFU_MAX_TREE || C > CONFU_MAX_TREE || V > 262144) return CONFU_ERR_UNSUPPORTED;
     if (B == 0) return CONFU_OK;
     if (!target_logits || !tokens || !parent || !accept_len || !path || !next_token) return CONFU_ERR_ARG;
     if (C > 0 && !con_owner) return CONFU_ERR_ARG;

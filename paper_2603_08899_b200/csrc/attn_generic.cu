@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(128) attention_generic_kernel(
             if (i < S_vis) { kp = ks + ((size_t)i * Hkv + g) * D; vis = true; }
             else {
                 const int64_t slot = i - S_vis;
-                vis = slot < P || ((mask >> (slot - P)) & 1ull);
+                const int64_t j = slot - P;              // >= 0: the slot of query row j
+                vis = j < 0 || (j < dm.T ? (int)((mask >> j) & 1ull) : (j == r));
                 kp = kc + ((size_t)(base + slot) * Hkv + g) * D;
             }
             if (vis) {

@@ -59,6 +59,7 @@ struct Params {
     float* lse;
     int32_t* status;
     int n_mt;            // M tiles in use (R > 32 ? 2 : 1)
+    int n_rg;            // groups of 64 query rows (R > 64 ? 2 : 1); a pair = (sequence, kv head, row group)
     int G;
     float c;             // sm_scale * log2(e)
 };
@@ -197,7 +198,7 @@ constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
 
 // ------------------------------------------------------------------------------------ work list
 struct Segment {
-    int b, g;
+    int b, g, rg;      // sequence, kv head, group of 64 query rows
     int t0, t1;        // tiles [t0, t1) of this pair
     int nt, nkt;       // tiles of the pair; key tiles (the soft-prompt tile, if any, is tile nkt)
     int64_t P;         // prefix length
@@ -238,7 +239,9 @@ struct Walker {
             if (t1 <= t0) continue;                    // the share ended inside this pair's overhead zone
             s.b = lo;
             s.nt = nt;
-            s.g = (int)(local / cost);
+            const int pair = (int)(local / cost);       // pairs of a sequence: kv head major, row group minor
+            s.g = pair / prm.n_rg;
+            s.rg = pair % prm.n_rg;
             s.t0 = t0;
             s.t1 = t1;
             s.nkt = nt - (prm.d.S > 0 ? 1 : 0);
@@ -313,7 +316,7 @@ __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanVi
                 mbar_arrive_expect_tx(&sh.q_full, 2u * prm.n_mt * q_box_bytes);
                 for (int mt = 0; mt < prm.n_mt; ++mt)
                     for (int kb = 0; kb < 2; ++kb)
-                        tma_load_3d(sh.q + (mt * 2 + kb) * kHalfTile, q_map, &sh.q_full, kb * 64, s.g * prm.G, s.b * R + 32 * mt);
+                        tma_load_3d(sh.q + (mt * 2 + kb) * kHalfTile, q_map, &sh.q_full, kb * 64, s.g * prm.G, s.b * R + kGroupRows * s.rg + 32 * mt);
             }
             prev = cur;
             have_prev = true;
@@ -409,10 +412,15 @@ __device__ __forceinline__ void visible_bits(const Segment& s, int t, int R, int
     unsigned __int128 v = 0;
     if (off >= 128) v = ~(unsigned __int128)0;
     else if (off > 0) v = (((unsigned __int128)1) << off) - 1;
-    // tree part: bit j of mask at position off + j
-    const unsigned __int128 m = (unsigned __int128)(R >= 64 ? mask : (mask & ((1ull << R) - 1)));
+    // tree rows' slots: bit j of mask at position off + j; a contemplate row's own slot at off + r
+    const unsigned __int128 m = (unsigned __int128)mask;
     if (off >= 0) { if (off < 128) v |= m << off; }
     else if (off > -64) v |= m >> (-off);
+    if (r >= T) {
+        const int64_t self = off + r;
+        if (self >= 0 && self < 128) v |= ((unsigned __int128)1) << self;
+    }
+    (void)R;
     lo = (uint64_t)v;
     hi = (uint64_t)(v >> 64);
 }
@@ -457,14 +465,15 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
     const uint32_t s_addr = tmem + lane_base + t * 128;
     const uint32_t o_addr = tmem + lane_base + 256 + t * 128;
     const int G = prm.G, T = prm.d.T, R = prm.d.T + prm.d.C, S = prm.d.S, Hq = prm.d.Hq;
-    const int r = 32 * t + lane_row / G, hl = lane_row % G;
-    const bool row_valid = lane_row < 32 * G && r < R;
+    const int hl = lane_row % G;
     const float c = prm.c;
 
     Walker w(pv, prm, blockIdx.x);
     Segment s;
     uint32_t n_s = 0, seg = 0;
     while (w.next(s)) {
+        const int r = kGroupRows * s.rg + 32 * t + lane_row / G;            // query row of this thread in this pair
+        const bool row_valid = lane_row < 32 * G && r < R;
         const uint64_t mask = row_valid ? pv.mask[(size_t)s.b * kMaxRows + r] : 0ull;
         float m_ref = -INFINITY, l = 0.f;
         for (int tile = s.t0; tile < s.t1; ++tile) {
@@ -643,19 +652,21 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
 {
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
     const int pair = blockIdx.x, t = blockIdx.y;
-    const int b = pair / prm.d.Hkv, g = pair % prm.d.Hkv;
+    // pairs: sequence major, then kv head, then row group
+    const int per_seq = prm.d.Hkv * prm.n_rg;
+    const int b = pair / per_seq, g = (pair % per_seq) / prm.n_rg, rg = pair % prm.n_rg;
     const int nt = pv.tiles[b];
     if (nt == 0 || t >= prm.n_mt) return;
     const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
     // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
-    const int64_t F = pv.tile_base[b] + (int64_t)g * (nt + kPairOverheadTiles) + kPairOverheadTiles;
+    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
     const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
     if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
     const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t slot_floats = partial_slot_bytes() / sizeof(float);
     for (int lane_row = blockIdx.z * 32 + warp; lane_row < min(32 * G, (int)blockIdx.z * 32 + 32); lane_row += 8) {
-        const int r = 32 * t + lane_row / G, hl = lane_row % G;
+        const int r = kGroupRows * rg + 32 * t + lane_row / G, hl = lane_row % G;
         if (r >= R) break;
         const int row = t * 128 + lane_row;
         float M = -INFINITY;
@@ -750,6 +761,7 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     prm.lse = lse;
     prm.status = status;
     prm.n_mt = R > 32 ? 2 : 1;
+    prm.n_rg = (R + kGroupRows - 1) / kGroupRows;
     prm.G = G;
     prm.c = (d.sm_scale != 0.f ? d.sm_scale : 1.f / sqrtf((float)d.D)) * 1.4426950408889634f;
     const size_t smem = sizeof(SharedStorage) + 1024;
@@ -762,7 +774,7 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     attention_tc_kernel<<<ctx->sm_count, kThreads, smem, st>>>(q_map, k_map, v_map, ks_map, vs_map, prm);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    combine_kernel<<<dim3(d.B * d.Hkv, prm.n_mt, 4), 256, 0, st>>>(prm);
+    combine_kernel<<<dim3(d.B * d.Hkv * prm.n_rg, prm.n_mt, 4), 256, 0, st>>>(prm);
     return cudaGetLastError();
 }
 

@@ -9,14 +9,17 @@
 
 namespace confu {
 
-constexpr int kMaxRows = CONFU_MAX_ROWS;        // R = T + C <= 64: one 64-bit mask word per row
+constexpr int kMaxRows = CONFU_MAX_ROWS;        // R = T + C <= 128
+constexpr int kMaxTree = CONFU_MAX_TREE;        // T <= 64: one 64-bit word of visible tree slots per row
+constexpr int kGroupRows = 64;                  // query rows the tensor-core kernel handles per pass over a pair's keys
 constexpr int kPathLen = CONFU_MAX_DEPTH + 1;
 constexpr int kTileKeys = 128;                  // keys per attention tile (tensor-core path)
 
 // ---------------------------------------------------------------------------
 // Plan buffer (device).  Built once per step by plan_kernel, read by every layer.
 //   PlanHeader
-//   uint64 mask[B][64]        bit j of mask[b][r]: row r sees tree slot j
+//   uint64 mask[B][128]       bit j < T of mask[b][r]: row r sees the slot of tree row j.  (A contemplate
+//                             row also sees its own slot and no other contemplate row's: not stored.)
 //   int32  bad[B]             non-zero: malformed tree, sequence skipped
 //   int32  tiles[B]           key tiles of one (sequence, kv head) pair, soft-prompt tile included
 //   int64  tile_base[B + 1]   position of sequence b's first pair on the flat cost line (exclusive scan)

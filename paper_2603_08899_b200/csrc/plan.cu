@@ -2,7 +2,8 @@
 //
 // Mask rule (tree attention over a token tree, with one contemplate token hung on a node's
 // branch): a tree row sees itself and its ancestors; a contemplate row sees itself, its owner
-// and the owner's ancestors.  Bit j of mask[b][r] says "row r sees tree slot j".
+// and the owner's ancestors.  Bit j < T of mask[b][r] says "row r sees the slot of tree row j";
+// that a contemplate row sees its own slot (and no other contemplate row's) is implied.
 #include "common.cuh"
 
 namespace confu {
@@ -15,11 +16,11 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
 {
     const int B = d.B, T = d.T, C = d.C, R = d.T + d.C;
     PlanView pv = plan_view(plan_raw, B);
-    __shared__ int s_bad[4];
-    __shared__ uint64_t s_mask[4][kMaxRows];
-    const int grp = threadIdx.x >> 6, r = threadIdx.x & 63;
+    __shared__ int s_bad[2];
+    __shared__ uint64_t s_mask[2][kMaxTree];
+    const int grp = threadIdx.x >> 7, r = threadIdx.x & 127;     // two sequences at a time, one thread per row
 
-    for (int b0 = 0; b0 < B; b0 += 4) {
+    for (int b0 = 0; b0 < B; b0 += 2) {
         const int b = b0 + grp;
         if (r == 0) s_bad[grp] = 0;
         __syncthreads();
@@ -36,29 +37,22 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
             if (code) atomicMax(&s_bad[grp], code == CONFU_ST_BAD_PARENT ? 2 : 1);
         }
         __syncthreads();
-        if (b < B) {
-            const int bad = s_bad[grp];
+        if (b < B && r < T) {
+            // a tree row sees itself and its ancestors
             const int32_t* par = parent + (size_t)b * T;
-            uint64_t m = 0;
-            if (r < T) {
-                m = 1ull << r;
-                if (!bad) {
-                    int a = par[r];
-                    for (int it = 0; it < T && a >= 0; ++it) { m |= 1ull << a; a = par[a]; }
-                }
-                s_mask[grp][r] = m;
+            uint64_t m = 1ull << r;
+            if (!s_bad[grp]) {
+                int a = par[r];
+                for (int it = 0; it < T && a >= 0; ++it) { m |= 1ull << a; a = par[a]; }
             }
-            __syncwarp();
+            s_mask[grp][r] = m;
         }
         __syncthreads();
         if (b < B) {
             const int bad = s_bad[grp];
             uint64_t m = 0;
             if (r < T) m = s_mask[grp][r];
-            else if (r < R) {
-                m = 1ull << r;
-                if (!bad) m |= s_mask[grp][con_owner[(size_t)b * C + (r - T)]];
-            }
+            else if (r < R && !bad) m = s_mask[grp][con_owner[(size_t)b * C + (r - T)]];   // owner and its ancestors (+ its own slot, implied)
             pv.mask[(size_t)b * kMaxRows + r] = m;
             if (r == 0) {
                 const int code = bad == 2 ? CONFU_ST_BAD_PARENT : (bad == 1 ? CONFU_ST_BAD_OWNER : 0);
@@ -74,7 +68,8 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
         int64_t acc = 0;
         for (int b = 0; b < B; ++b) {
             pv.tile_base[b] = acc;
-            if (pv.tiles[b] > 0) acc += (int64_t)(pv.tiles[b] + kPairOverheadTiles) * d.Hkv;
+            // one pair per (kv head, group of 64 query rows)
+            if (pv.tiles[b] > 0) acc += (int64_t)(pv.tiles[b] + kPairOverheadTiles) * d.Hkv * ((R + kGroupRows - 1) / kGroupRows);
         }
         pv.tile_base[B] = acc;
         PlanHeader h;

@@ -66,6 +66,15 @@ CONFIGS = {
                             prefix=(512, 16384), tree="random", kv_dtype=torch.bfloat16,
                             logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",
                             temperatures=(1.0,), seed=5),
+    # one contemplate row per draft node (the verification forward of Sec. 3.1 processes 2T rows)
+    "llama8b_2t": VerifyConfig("llama8b_2t", B=1, L=32, Hq=32, Hkv=8, D=128, T=60, C=60, S=16, V=128256,
+                               prefix=4096, tree="random", kv_dtype=torch.bfloat16,
+                               logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",
+                               temperatures=(1.0,), seed=6),
+    "batch32_2t": VerifyConfig("batch32_2t", B=32, L=32, Hq=32, Hkv=8, D=128, T=60, C=60, S=16, V=128256,
+                               prefix=(512, 16384), tree="random", kv_dtype=torch.bfloat16,
+                               logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",
+                               temperatures=(1.0,), seed=7),
 }
 
 

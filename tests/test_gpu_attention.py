@@ -42,6 +42,13 @@ CASES = {
     "bf16_paper_sized_30_30": _cfg(B=1, T=30, C=30, S=16, prefix=1000, max_depth=7, fanout=(1, 4), seed=46),
     "bf16_exact_tile_multiple": _cfg(B=1, T=12, C=4, prefix=256 - 16, seed=47),
     "bf16_one_past_tile": _cfg(B=1, T=12, C=4, prefix=256 - 15, seed=48),
+    # more than 64 query rows: one contemplate row per tree node (R = 2T), two groups of 64 rows
+    "bf16_one_contemplate_per_node_60_60": _cfg(B=2, T=60, C=60, S=16, prefix=(130, 520), max_depth=7, fanout=(1, 4), seed=49),
+    "bf16_rows_65": _cfg(T=33, C=32, S=16, prefix=(60, 200), max_depth=7, fanout=(1, 4), seed=50),
+    "bf16_g3_rows_80": _cfg(Hq=6, Hkv=2, T=40, C=40, prefix=(1, 300), max_depth=7, fanout=(1, 4), seed=51),
+    "bf16_rows_128_chain": _cfg(B=1, T=64, C=64, S=16, tree="chain", prefix=257, seed=52),
+    "fp32_rows_100": _cfg(kv_dtype=torch.float32, T=50, C=50, prefix=(10, 150), max_depth=7, fanout=(1, 4), seed=53),
+    "bf16_d64_rows_90": _cfg(D=64, T=45, C=45, prefix=(10, 150), max_depth=7, fanout=(1, 4), seed=54),
 }
 
 
@@ -56,7 +63,8 @@ def test_attention_matches_oracle(gpu, name, use_plan):
     H.assert_attention_close(out, lse, want, want_lse, cfg.kv_dtype, name)
 
 
-@pytest.mark.parametrize("name", ["bf16_full_rows", "bf16_g3", "bf16_paper_sized_30_30", "fp32_d128_ragged"])
+@pytest.mark.parametrize("name", ["bf16_full_rows", "bf16_g3", "bf16_paper_sized_30_30", "fp32_d128_ragged",
+                                  "bf16_one_contemplate_per_node_60_60", "bf16_g3_rows_80", "fp32_rows_100"])
 def test_mask_sensitivity_with_boosted_tree_keys(gpu, name):
     """With the tree slots' keys scaled up the tree columns dominate the softmax, so a wrong
     ancestor bit moves the output far beyond tolerance even behind a long prefix."""
@@ -124,8 +132,10 @@ def test_host_side_argument_errors(gpu):
     with pytest.raises(cb.ConfuError) as e:
         H.gpu_attention(gpu, inputs.scaled(cfg, D=96), t, seq_start, plen, parent, owner, n_slots)
     assert e.value.code == -2
-    dims = H.dims_of(inputs.scaled(cfg, T=62, C=3))
-    assert cb.lib().confu_workspace_bytes(gpu.ctx, __import__("ctypes").byref(dims)) == 0      # R > 64 unsupported
+    dims = H.dims_of(inputs.scaled(cfg, T=65, C=3))
+    assert cb.lib().confu_workspace_bytes(gpu.ctx, __import__("ctypes").byref(dims)) == 0      # T > 64 unsupported
+    dims = H.dims_of(inputs.scaled(cfg, T=64, C=64))
+    assert cb.lib().confu_workspace_bytes(gpu.ctx, __import__("ctypes").byref(dims)) > 0       # R = 128 is the limit
     # unaligned q pointer
     dims = H.dims_of(cfg)
     gpu.ensure_ws(dims)

@@ -65,7 +65,7 @@ def test_tiny_config_full():
         assert exact + border == 1
 
 
-@pytest.mark.parametrize("name,prefix", [("llama3b", 700), ("llama8b", 900), ("qwen4b", 1100)])
+@pytest.mark.parametrize("name,prefix", [("llama3b", 700), ("llama8b", 900), ("qwen4b", 1100), ("llama8b_2t", 600)])
 def test_llm_shaped_steps_reduced_prefix(name, prefix):
     """Real head counts, tree sizes and vocabularies; prefix and layer count cut so the oracle
     finishes in seconds; still several key tiles and a ragged tail."""
@@ -83,7 +83,7 @@ def test_batched_ragged_step_reduced():
     assert exact + border == cfg.B and border <= 1
 
 
-@pytest.mark.parametrize("name", ["llama3b", "llama8b", "qwen4b", "batch32"])
+@pytest.mark.parametrize("name", ["llama3b", "llama8b", "qwen4b", "batch32", "llama8b_2t"])
 def test_full_size_attention_on_sampled_rows(name):
     """The full-size workload of the benchmark, one layer, in the launch configuration the
     benchmark times; the oracle recomputes a sample of output rows one by one."""
