@@ -138,3 +138,60 @@ def test_full_size_acceptance(name):
     exact, border = H.compare_accept(got, want)
     assert exact + border == cfg.B and border <= 1
     g.close()
+
+
+def test_two_chained_steps_through_compaction_and_append():
+    """Step 1 (attention, acceptance, compaction), then a second step on the compacted cache: the new
+    tree's K/V rows are placed behind the new prefix with confu_kv_append and attention runs with
+    new_prefix_len as the prefix.  The oracle replays the same two steps on host copies."""
+    cfg = inputs.scaled(inputs.CONFIGS["batch32"], B=4, prefix=(40, 500), L=2)
+    parent, owner, plen, seq_start, n_slots, lt, tl, dl, tok, u = _build(cfg, cfg.L, 1.0)
+    # leave room behind every sequence for the second step's rows: rebuild the layout with slack
+    seq_start, n_slots = inputs.cache_layout(cfg, plen + 16)
+    lt = [inputs.layer_tensors(cfg, l, n_slots, device="cuda") for l in range(cfg.L)]
+    host = [{k: (None if v is None else v.cpu().clone()) for k, v in t.items()} for t in lt]
+    step = VerifyStep(cfg, n_slots)
+    outs = [torch.empty_like(t["q"]) for t in lt]
+    step.bind([t["q"] for t in lt], [t["k_cache"] for t in lt], [t["v_cache"] for t in lt],
+              [t["k_soft"] for t in lt], [t["v_soft"] for t in lt], outs, seq_start.cuda(), plen.cuda(),
+              parent.cuda(), owner.cuda(), tl, dl, tok.cuda(), u.cuda())
+    step.run(1.0)
+    torch.cuda.synchronize()
+    assert (step.status == 0).all()
+    # ---- oracle: step 1 acceptance and compaction on the host copies
+    want = ref.tree_accept(tl.cpu(), dl.cpu(), tok, parent, owner, u, temperature=1.0)
+    got = {"accept_len": step.accept_len.cpu(), "path": step.path.cpu(), "next_token": step.next_token.cpu(),
+           "future_row": step.future_row.cpu(), "counters": step.counters.cpu(), "status": step.status.cpu()}
+    exact, border = H.compare_accept(got, want)
+    kh, vh = [h["k_cache"] for h in host], [h["v_cache"] for h in host]
+    # replay the GPU's accepted path (it equals the oracle's unless a borderline decision differed)
+    new_len_host = ref.kv_compact(kh, vh, seq_start, plen, got["accept_len"], got["path"])
+    assert step.new_prefix_len.cpu().tolist() == new_len_host.tolist()
+    # ---- step 2: a fresh tree on the compacted cache
+    cfg2 = inputs.scaled(cfg, seed=cfg.seed + 77)
+    parent2, owner2 = inputs.trees(cfg2)
+    g = torch.Generator().manual_seed(123)
+    new_plen = step.new_prefix_len.clone()
+    for l in range(cfg.L):
+        q2 = torch.randn(cfg.B, cfg.R, cfg.Hq, cfg.D, generator=g).to(cfg.kv_dtype)
+        k_rows = torch.randn(cfg.B, cfg.R, cfg.Hkv, cfg.D, generator=g).to(cfg.kv_dtype)
+        v_rows = torch.randn(cfg.B, cfg.R, cfg.Hkv, cfg.D, generator=g).to(cfg.kv_dtype)
+        cb.confu_kv_append(step.ctx, step.dims, k_rows.cuda(), v_rows.cuda(), lt[l]["k_cache"], lt[l]["v_cache"],
+                           step.seq_start, new_plen)
+        out2 = torch.empty_like(lt[l]["q"])
+        lse2 = torch.empty(cfg.B, cfg.R, cfg.Hq, dtype=torch.float32, device="cuda")
+        st2 = torch.zeros(cfg.B, dtype=torch.int32, device="cuda")
+        cb.confu_tree_attention(step.ctx, step.dims, q2.cuda(), lt[l]["k_cache"], lt[l]["v_cache"], n_slots,
+                                step.seq_start, new_plen, lt[l]["k_soft"], lt[l]["v_soft"], parent2.cuda(),
+                                owner2.cuda(), None, out2, lse2, st2)
+        torch.cuda.synchronize()
+        assert (st2 == 0).all()
+        # host: same append on the compacted host cache, then the oracle
+        for b in range(cfg.B):
+            lo = int(seq_start[b]) + int(new_len_host[b])
+            kh[l][lo:lo + cfg.R] = k_rows[b]
+            vh[l][lo:lo + cfg.R] = v_rows[b]
+        w, wl, _ = ref.tree_attention(q2, kh[l], vh[l], seq_start, new_len_host, host[l]["k_soft"], host[l]["v_soft"],
+                                      parent2, owner2)
+        H.assert_attention_close(out2.cpu(), lse2.cpu(), w, wl, cfg.kv_dtype, f"second step layer {l}")
+    step.close()
