@@ -102,6 +102,18 @@ int confu_destroy(confu_ctx* ctx);
 size_t confu_workspace_bytes(const confu_ctx* ctx, const confu_dims* dims);
 int confu_set_workspace(confu_ctx* ctx, void* device_ptr, size_t bytes);
 
+/*
+ * Paged pools.  With a block table set, every layer's cache pool is read as pages of 128 slots:
+ * slot s of sequence b (s = 0 is its first prefix token; the R query rows follow the prefix) lives
+ * in page block_table[b][s / 128] at offset s % 128, i.e. at pool slot 128 * page + s % 128.
+ * block_table: DEVICE int32 [B][max_pages], with at least ceil((prefix_len[b] + R) / 128) valid
+ * page ids per sequence; read by every later call until it is cleared (NULL); seq_start is then
+ * ignored and may be NULL, and n_slots must be a whole number of pages.  The paper has no cache
+ * layout (Sec. 3.1 only says the K/V of accepted tokens are kept); pages of one key tile are what
+ * serving engines use.
+ */
+int confu_set_paging(confu_ctx* ctx, const int32_t* block_table, int32_t max_pages);
+
 const char* confu_status_string(int code);      /* host return codes and device status codes */
 const char* confu_last_cuda_error(const confu_ctx* ctx);
 

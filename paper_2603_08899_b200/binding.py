@@ -22,7 +22,7 @@ EXPORTS = [
     "confu_create", "confu_destroy", "confu_workspace_bytes", "confu_set_workspace", "confu_status_string",
     "confu_last_cuda_error", "confu_plan_bytes", "confu_tree_plan", "confu_tree_attention",
     "confu_accept_workspace_bytes", "confu_tree_accept", "confu_kv_compact", "confu_kv_append",
-    "confu_tree_accept_static_max_rows", "confu_tree_accept_static",
+    "confu_tree_accept_static_max_rows", "confu_tree_accept_static", "confu_set_paging",
 ]
 
 
@@ -49,7 +49,7 @@ def lib():
         L.confu_status_string.restype = C.c_char_p
         L.confu_last_cuda_error.restype = C.c_char_p
         for n in ("confu_create", "confu_destroy", "confu_set_workspace", "confu_tree_plan", "confu_tree_attention",
-                  "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static"):
+                  "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static", "confu_set_paging"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -108,6 +108,11 @@ def confu_workspace_bytes(ctx, dims):
 def confu_set_workspace(ctx, tensor):
     nbytes = 0 if tensor is None else tensor.numel() * tensor.element_size()
     _check("confu_set_workspace", lib().confu_set_workspace(ctx, _ptr(tensor), C.c_size_t(nbytes)))
+
+
+def confu_set_paging(ctx, block_table, max_pages=0):
+    """block_table: int32 CUDA tensor [B, max_pages] (kept alive by the caller), or None for packed pools."""
+    _check("confu_set_paging", lib().confu_set_paging(ctx, _ptr(block_table), C.c_int32(max_pages)))
 
 
 def confu_plan_bytes(ctx, dims):

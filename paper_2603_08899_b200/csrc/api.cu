@@ -42,7 +42,7 @@ size_t ws_total(const confu_ctx* ctx, const confu_dims* d)
 namespace confu {
 bool tc_attention_supported(const confu_dims& d);
 cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
-                                const void* v_cache, int64_t n_slots, const int64_t* seq_start,
+                                const void* v_cache, int64_t n_slots, const SlotMap& map,
                                 const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
                                 void* partials, void* out, float* lse, int32_t* status, cudaStream_t st);
 }  // namespace confu
@@ -59,6 +59,8 @@ int confu_create(confu_ctx** out, int device)
     c->workspace = nullptr;
     c->workspace_bytes = 0;
     c->dev_flags = nullptr;
+    c->block_table = nullptr;
+    c->max_pages = 0;
     c->last_error = cudaSuccess;
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
@@ -92,6 +94,15 @@ int confu_set_workspace(confu_ctx* ctx, void* device_ptr, size_t bytes)
     if (device_ptr && misaligned(device_ptr)) return CONFU_ERR_ALIGN;
     ctx->workspace = device_ptr;
     ctx->workspace_bytes = device_ptr ? bytes : 0;
+    return CONFU_OK;
+}
+
+int confu_set_paging(confu_ctx* ctx, const int32_t* block_table, int32_t max_pages)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    if (block_table && max_pages <= 0) return CONFU_ERR_ARG;
+    ctx->block_table = block_table;
+    ctx->max_pages = block_table ? max_pages : 0;
     return CONFU_OK;
 }
 
@@ -135,7 +146,7 @@ int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims, const int64_t* seq_s
     int rc = check_dims(dims);
     if (rc != CONFU_OK) return rc;
     if (!plan) return CONFU_ERR_ARG;
-    if (dims->B > 0 && (!seq_start || !prefix_len || !parent || (dims->C > 0 && !con_owner))) return CONFU_ERR_ARG;
+    if (dims->B > 0 && (!prefix_len || !parent || (dims->C > 0 && !con_owner))) return CONFU_ERR_ARG;
     if (misaligned(plan)) return CONFU_ERR_ALIGN;
     cudaError_t e = launch_plan(ctx, *dims, seq_start, prefix_len, parent, con_owner, plan, status, (cudaStream_t)stream);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
@@ -150,7 +161,10 @@ int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims, const void* q, 
     int rc = check_dims(dims);
     if (rc != CONFU_OK) return rc;
     if (dims->B == 0) return CONFU_OK;
-    if (!q || !k_cache || !v_cache || !seq_start || !prefix_len || !out || n_slots <= 0) return CONFU_ERR_ARG;
+    if (!q || !k_cache || !v_cache || !prefix_len || !out || n_slots <= 0) return CONFU_ERR_ARG;
+    if (!ctx->block_table && !seq_start) return CONFU_ERR_ARG;
+    if (ctx->block_table && n_slots % kTileKeys != 0) return CONFU_ERR_SHAPE;      // a paged pool is whole pages
+    const SlotMap map = {seq_start, ctx->block_table, ctx->max_pages};
     if (dims->S > 0 && (!k_soft || !v_soft)) return CONFU_ERR_ARG;
     if (!plan && (!parent || (dims->C > 0 && !con_owner))) return CONFU_ERR_ARG;
     if (misaligned(q) || misaligned(k_cache) || misaligned(v_cache) || misaligned(out) || misaligned(k_soft) ||
@@ -168,10 +182,10 @@ int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims, const void* q, 
     }
     cudaError_t e;
     if (tc_attention_supported(*dims))
-        e = launch_attention_tc(ctx, *dims, q, k_cache, v_cache, n_slots, seq_start, prefix_len, k_soft, v_soft,
+        e = launch_attention_tc(ctx, *dims, q, k_cache, v_cache, n_slots, map, prefix_len, k_soft, v_soft,
                                 use_plan, ws + ws_partial_offset(dims), out, lse, status, st);
     else
-        e = launch_attention_generic(ctx, *dims, q, k_cache, v_cache, seq_start, prefix_len, k_soft, v_soft, use_plan,
+        e = launch_attention_generic(ctx, *dims, q, k_cache, v_cache, map, prefix_len, k_soft, v_soft, use_plan,
                                      out, lse, st);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
 }
@@ -217,10 +231,12 @@ int confu_kv_compact(confu_ctx* ctx, const confu_dims* dims, int32_t n_layers, v
     if (rc != CONFU_OK) return rc;
     if (n_layers < 0) return CONFU_ERR_ARG;
     if (dims->B == 0) return CONFU_OK;
-    if (!seq_start || !prefix_len || !accept_len || !path) return CONFU_ERR_ARG;
+    if (!prefix_len || !accept_len || !path) return CONFU_ERR_ARG;
+    if (!ctx->block_table && !seq_start) return CONFU_ERR_ARG;
+    const SlotMap map = {seq_start, ctx->block_table, ctx->max_pages};
     if (n_layers > 0 && (!k_cache_layers || !v_cache_layers)) return CONFU_ERR_ARG;
     const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : 4);
-    cudaError_t e = launch_compact(ctx, dims->B, n_layers, row_bytes, k_cache_layers, v_cache_layers, seq_start,
+    cudaError_t e = launch_compact(ctx, dims->B, n_layers, row_bytes, k_cache_layers, v_cache_layers, map,
                                    prefix_len, accept_len, path, new_prefix_len, status, (cudaStream_t)stream);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
 }
@@ -232,10 +248,12 @@ int confu_kv_append(confu_ctx* ctx, const confu_dims* dims, const void* k_rows, 
     int rc = check_dims(dims);
     if (rc != CONFU_OK) return rc;
     if (dims->B == 0) return CONFU_OK;
-    if (!k_rows || !v_rows || !k_cache || !v_cache || !seq_start || !prefix_len) return CONFU_ERR_ARG;
+    if (!k_rows || !v_rows || !k_cache || !v_cache || !prefix_len) return CONFU_ERR_ARG;
+    if (!ctx->block_table && !seq_start) return CONFU_ERR_ARG;
+    const SlotMap map = {seq_start, ctx->block_table, ctx->max_pages};
     if (misaligned(k_rows) || misaligned(v_rows) || misaligned(k_cache) || misaligned(v_cache)) return CONFU_ERR_ALIGN;
     const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : 4);
-    cudaError_t e = launch_append(dims->B, dims->T + dims->C, row_bytes, k_rows, v_rows, k_cache, v_cache, seq_start,
+    cudaError_t e = launch_append(dims->B, dims->T + dims->C, row_bytes, k_rows, v_rows, k_cache, v_cache, map,
                                   prefix_len, (cudaStream_t)stream);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
 }

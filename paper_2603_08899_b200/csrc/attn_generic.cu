@@ -11,7 +11,7 @@ namespace confu {
 template <typename T, int D>
 __global__ void __launch_bounds__(128) attention_generic_kernel(
     confu_dims dm, const T* __restrict__ q, const T* __restrict__ kc, const T* __restrict__ vc,
-    const int64_t* __restrict__ seq_start, const int32_t* __restrict__ prefix_len, const T* __restrict__ ks,
+    const SlotMap map, const int32_t* __restrict__ prefix_len, const T* __restrict__ ks,
     const T* __restrict__ vs, const void* plan_raw, T* __restrict__ out, float* __restrict__ lse)
 {
     constexpr int NT = 128;
@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(128) attention_generic_kernel(
         return;
     }
     const uint64_t mask = pv.mask[(size_t)b * kMaxRows + r];
-    const int64_t P = prefix_len[b], base = seq_start[b];
+    const int64_t P = prefix_len[b];
     const int S_vis = (r >= dm.T) ? dm.S : 0;
     const int64_t n = S_vis + P + R;
     const float scale = dm.sm_scale != 0.f ? dm.sm_scale : rsqrtf((float)D);
@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(128) attention_generic_kernel(
                 const int64_t slot = i - S_vis;
                 const int64_t j = slot - P;              // >= 0: the slot of query row j
                 vis = j < 0 || (j < dm.T ? (int)((mask >> j) & 1ull) : (j == r));
-                kp = kc + ((size_t)(base + slot) * Hkv + g) * D;
+                kp = kc + ((size_t)pool_slot(map, b, slot) * Hkv + g) * D;
             }
             if (vis) {
                 float a = 0.f;
@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(128) attention_generic_kernel(
                 if (pj == 0.f) continue;
                 const int64_t ii = c0 + j;
                 const T* vp = (ii < S_vis) ? vs + ((size_t)ii * Hkv + g) * D
-                                           : vc + ((size_t)(base + ii - S_vis) * Hkv + g) * D;
+                                           : vc + ((size_t)pool_slot(map, b, ii - S_vis) * Hkv + g) * D;
                 acc = fmaf(pj, to_f32(vp[tid]), acc);
             }
         }
@@ -102,28 +102,28 @@ __global__ void __launch_bounds__(128) attention_generic_kernel(
 
 template <typename T>
 static cudaError_t launch_t(const confu_dims& d, const void* q, const void* kc, const void* vc,
-                            const int64_t* seq_start, const int32_t* prefix_len, const void* ks, const void* vs,
+                            const SlotMap& map, const int32_t* prefix_len, const void* ks, const void* vs,
                             const void* plan, void* out, float* lse, cudaStream_t st)
 {
     dim3 grid(d.T + d.C, d.Hq, d.B);
     if (d.B == 0) return cudaSuccess;
     if (d.D == 64)
-        attention_generic_kernel<T, 64><<<grid, 128, 0, st>>>(d, (const T*)q, (const T*)kc, (const T*)vc, seq_start,
+        attention_generic_kernel<T, 64><<<grid, 128, 0, st>>>(d, (const T*)q, (const T*)kc, (const T*)vc, map,
                                                               prefix_len, (const T*)ks, (const T*)vs, plan, (T*)out, lse);
     else
-        attention_generic_kernel<T, 128><<<grid, 128, 0, st>>>(d, (const T*)q, (const T*)kc, (const T*)vc, seq_start,
+        attention_generic_kernel<T, 128><<<grid, 128, 0, st>>>(d, (const T*)q, (const T*)kc, (const T*)vc, map,
                                                                prefix_len, (const T*)ks, (const T*)vs, plan, (T*)out, lse);
     return cudaGetLastError();
 }
 
 cudaError_t launch_attention_generic(const Ctx*, const confu_dims& d, const void* q, const void* k_cache,
-                                     const void* v_cache, const int64_t* seq_start, const int32_t* prefix_len,
+                                     const void* v_cache, const SlotMap& map, const int32_t* prefix_len,
                                      const void* k_soft, const void* v_soft, const void* plan, void* out,
                                      float* lse, cudaStream_t st)
 {
     if (d.kv_dtype == CONFU_F32)
-        return launch_t<float>(d, q, k_cache, v_cache, seq_start, prefix_len, k_soft, v_soft, plan, out, lse, st);
-    return launch_t<__nv_bfloat16>(d, q, k_cache, v_cache, seq_start, prefix_len, k_soft, v_soft, plan, out, lse, st);
+        return launch_t<float>(d, q, k_cache, v_cache, map, prefix_len, k_soft, v_soft, plan, out, lse, st);
+    return launch_t<__nv_bfloat16>(d, q, k_cache, v_cache, map, prefix_len, k_soft, v_soft, plan, out, lse, st);
 }
 
 }  // namespace confu

@@ -51,7 +51,7 @@ struct SharedStorage {
 
 struct Params {
     confu_dims d;
-    const int64_t* seq_start;
+    SlotMap map;         // packed pool (seq_start) or paged pool (block table, pages of 128 slots = one key tile)
     const int32_t* prefix_len;
     const void* plan;
     float* partials;
@@ -202,7 +202,7 @@ struct Segment {
     int t0, t1;        // tiles [t0, t1) of this pair
     int nt, nkt;       // tiles of the pair; key tiles (the soft-prompt tile, if any, is tile nkt)
     int64_t P;         // prefix length
-    int64_t slot0;     // seq_start
+    int64_t slot0;     // packed pool: the sequence's first slot
     int part_slot;     // -1: the range covers the whole pair, write the output directly
 };
 
@@ -246,7 +246,7 @@ struct Walker {
             s.t1 = t1;
             s.nkt = nt - (prm.d.S > 0 ? 1 : 0);
             s.P = prm.prefix_len[lo];
-            s.slot0 = prm.seq_start[lo];
+            s.slot0 = prm.map.block_table ? 0 : prm.map.seq_start[lo];
             const bool whole = t0 == 0 && t1 == nt;
             s.part_slot = whole ? -1 : 2 * cta + (t1 < nt ? 1 : 0);
             return true;
@@ -307,7 +307,10 @@ __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanVi
             TileRef cur;
             cur.g = s.g;
             cur.soft = t >= s.nkt;
-            cur.z = cur.soft ? 0 : (int)(s.slot0 + (int64_t)t * kTileKeys);
+            // key tile t of a sequence is its slots 128 t .. 128 t + 127: one page of a paged pool
+            cur.z = cur.soft ? 0
+                  : prm.map.block_table ? prm.map.block_table[(size_t)s.b * prm.map.max_pages + t] * kTileKeys
+                                        : (int)(s.slot0 + (int64_t)t * kTileKeys);
             // the stage first (it carries the previous pair's last V tile, which must not wait for
             // the Q buffer), then, at the start of a pair, its Q (both M tiles, two 64-wide halves each)
             if (!fill(&cur)) return;
@@ -739,7 +742,7 @@ bool tc_attention_supported(const confu_dims& d)
 }
 
 cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
-                                const void* v_cache, int64_t n_slots, const int64_t* seq_start,
+                                const void* v_cache, int64_t n_slots, const SlotMap& map,
                                 const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
                                 void* partials, void* out, float* lse, int32_t* status, cudaStream_t st)
 {
@@ -753,7 +756,7 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     if (!ok) return cudaErrorInvalidValue;
     Params prm;
     prm.d = d;
-    prm.seq_start = seq_start;
+    prm.map = map;
     prm.prefix_len = prefix_len;
     prm.plan = plan;
     prm.partials = (float*)partials;

@@ -78,11 +78,26 @@ __host__ __device__ inline size_t partial_slot_bytes()
     return (size_t)kPartRows * kPartD * sizeof(float) + (size_t)kPartRows * 2 * sizeof(float);
 }
 
+// Where sequence b's slot s (0 = first prefix token) lives in a layer's pool: behind seq_start[b]
+// in a packed pool, or in page block_table[b][s / 128] of a paged pool (pages of kTileKeys slots).
+struct SlotMap {
+    const int64_t* seq_start;
+    const int32_t* block_table;    // [B][max_pages] page ids, or nullptr for a packed pool
+    int32_t max_pages;
+};
+__device__ __forceinline__ int64_t pool_slot(const SlotMap& m, int b, int64_t s)
+{
+    if (m.block_table) return (int64_t)m.block_table[(size_t)b * m.max_pages + (s >> 7)] * kTileKeys + (s & (kTileKeys - 1));
+    return m.seq_start[b] + s;
+}
+
 struct Ctx {
     int device;
     int sm_count;
     void* workspace;
     size_t workspace_bytes;
+    const int32_t* block_table;    // paged pools when set (confu_set_paging)
+    int32_t max_pages;
     int32_t* dev_flags;        // small device block owned by the context
     cudaError_t last_error;
 };
@@ -155,7 +170,7 @@ cudaError_t launch_plan(const Ctx* ctx, const confu_dims& d, const int64_t* seq_
                         cudaStream_t st);
 
 cudaError_t launch_attention_generic(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
-                                     const void* v_cache, const int64_t* seq_start, const int32_t* prefix_len,
+                                     const void* v_cache, const SlotMap& map, const int32_t* prefix_len,
                                      const void* k_soft, const void* v_soft, const void* plan, void* out,
                                      float* lse, cudaStream_t st);
 
@@ -167,11 +182,11 @@ cudaError_t launch_accept(const Ctx* ctx, int B, int T, int C, int V, int logit_
 size_t accept_workspace_bytes(int B, int T, int V);
 
 cudaError_t launch_compact(const Ctx* ctx, int B, int n_layers, int64_t row_bytes, void* const* k_layers,
-                           void* const* v_layers, const int64_t* seq_start, const int32_t* prefix_len,
+                           void* const* v_layers, const SlotMap& map, const int32_t* prefix_len,
                            const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len,
                            int32_t* status, cudaStream_t st);
 
 cudaError_t launch_append(int B, int R, int64_t row_bytes, const void* k_rows, const void* v_rows, void* k_cache,
-                          void* v_cache, const int64_t* seq_start, const int32_t* prefix_len, cudaStream_t st);
+                          void* v_cache, const SlotMap& map, const int32_t* prefix_len, cudaStream_t st);
 
 }  // namespace confu

@@ -15,7 +15,7 @@ constexpr int kCompactBatch = 8;
 
 __global__ void __launch_bounds__(128) compact_kernel(int n_layers, int64_t row_vecs, void* const* __restrict__ k_layers,
                                                       void* const* __restrict__ v_layers,
-                                                      const int64_t* __restrict__ seq_start,
+                                                      const SlotMap map,
                                                       const int32_t* __restrict__ prefix_len,
                                                       const int32_t* __restrict__ accept_len,
                                                       const int32_t* __restrict__ path,
@@ -29,16 +29,16 @@ __global__ void __launch_bounds__(128) compact_kernel(int n_layers, int64_t row_
         new_prefix_len[b] = prefix_len[b] + a + 1;
     if (a == 0 || col >= row_vecs) return;
     uint4* pool = reinterpret_cast<uint4*>(kv ? v_layers[layer] : k_layers[layer]);
-    const int64_t root = seq_start[b] + prefix_len[b];
+    const int64_t root = prefix_len[b];              // the root's slot, counted from the sequence's first
     const int32_t* pth = path + (size_t)b * kPathLen;
     for (int k0 = 1; k0 <= a; k0 += kCompactBatch) {
         uint4 buf[kCompactBatch];
 #pragma unroll
         for (int j = 0; j < kCompactBatch; ++j)
-            if (k0 + j <= a) buf[j] = pool[(root + pth[k0 + j]) * row_vecs + col];
+            if (k0 + j <= a) buf[j] = pool[pool_slot(map, b, root + pth[k0 + j]) * row_vecs + col];
 #pragma unroll
         for (int j = 0; j < kCompactBatch; ++j)
-            if (k0 + j <= a) pool[(root + k0 + j) * row_vecs + col] = buf[j];
+            if (k0 + j <= a) pool[pool_slot(map, b, root + k0 + j) * row_vecs + col] = buf[j];
     }
     (void)n_layers;
 }
@@ -46,26 +46,26 @@ __global__ void __launch_bounds__(128) compact_kernel(int n_layers, int64_t row_
 // cache[seq_start[b] + prefix_len[b] + r] = rows[b][r]  (K and V of the step's own query rows)
 __global__ void __launch_bounds__(128) append_kernel(int R, int64_t row_vecs, const uint4* __restrict__ k_rows,
                                                      const uint4* __restrict__ v_rows, uint4* __restrict__ k_cache,
-                                                     uint4* __restrict__ v_cache, const int64_t* __restrict__ seq_start,
+                                                     uint4* __restrict__ v_cache, const SlotMap map,
                                                      const int32_t* __restrict__ prefix_len)
 {
     const int r = blockIdx.x, b = blockIdx.y, kv = blockIdx.z;
     const uint4* src = (kv ? v_rows : k_rows) + ((size_t)b * R + r) * row_vecs;
-    uint4* dst = (kv ? v_cache : k_cache) + (size_t)(seq_start[b] + prefix_len[b] + r) * row_vecs;
+    uint4* dst = (kv ? v_cache : k_cache) + (size_t)pool_slot(map, b, (int64_t)prefix_len[b] + r) * row_vecs;
     for (int64_t c = threadIdx.x; c < row_vecs; c += blockDim.x) dst[c] = src[c];
 }
 
 cudaError_t launch_append(int B, int R, int64_t row_bytes, const void* k_rows, const void* v_rows, void* k_cache,
-                          void* v_cache, const int64_t* seq_start, const int32_t* prefix_len, cudaStream_t st)
+                          void* v_cache, const SlotMap& map, const int32_t* prefix_len, cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
     append_kernel<<<dim3(R, B, 2), 128, 0, st>>>(R, row_bytes / 16, (const uint4*)k_rows, (const uint4*)v_rows,
-                                                 (uint4*)k_cache, (uint4*)v_cache, seq_start, prefix_len);
+                                                 (uint4*)k_cache, (uint4*)v_cache, map, prefix_len);
     return cudaGetLastError();
 }
 
 cudaError_t launch_compact(const Ctx*, int B, int n_layers, int64_t row_bytes, void* const* k_layers,
-                           void* const* v_layers, const int64_t* seq_start, const int32_t* prefix_len,
+                           void* const* v_layers, const SlotMap& map, const int32_t* prefix_len,
                            const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len,
                            int32_t* /*status*/, cudaStream_t st)
 {
@@ -74,10 +74,10 @@ cudaError_t launch_compact(const Ctx*, int B, int n_layers, int64_t row_bytes, v
     // with no layers there is still new_prefix_len to write: one block row does it
     dim3 grid((unsigned)((row_vecs + 127) / 128), (unsigned)(n_layers > 0 ? 2 * n_layers : 1), (unsigned)B);
     if (n_layers == 0) {
-        compact_kernel<<<dim3(1, 1, B), 128, 0, st>>>(0, 0, k_layers, v_layers, seq_start, prefix_len, accept_len, path,
+        compact_kernel<<<dim3(1, 1, B), 128, 0, st>>>(0, 0, k_layers, v_layers, map, prefix_len, accept_len, path,
                                                        new_prefix_len);
     } else {
-        compact_kernel<<<grid, 128, 0, st>>>(n_layers, row_vecs, k_layers, v_layers, seq_start, prefix_len, accept_len,
+        compact_kernel<<<grid, 128, 0, st>>>(n_layers, row_vecs, k_layers, v_layers, map, prefix_len, accept_len,
                                              path, new_prefix_len);
     }
     return cudaGetLastError();
