@@ -615,11 +615,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     const uint32_t tmem = sh.tmem_base;
 
     if (warp < 8) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         const int t = warp >> 2;
         if (t < prm.n_mt) softmax_role(sh, prm, pv, tmem, t);
     } else {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
         if (warp == 8) {
             if ((threadIdx.x & 31) == 0) producer_role(sh, prm, pv, &q_map, &k_map, &v_map, &ks_map, &vs_map);
         } else if (warp == 9) {
