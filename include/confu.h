@@ -20,8 +20,7 @@
  *     aligned; the caller owns every buffer it passes, for the whole time the
  *     enqueued work runs;
  *   - work is enqueued on the given stream (a cudaStream_t passed as void*); no call
- *     synchronises the host with the device and none allocates device memory except
- *     confu_create / confu_destroy;
+ *     synchronises the host with the device and none allocates device memory;
  *   - data-dependent problems (a malformed tree, an out-of-range token, a
  *     non-finite logit, a bounded device-side wait that ran out) never trap: the
  *     kernels write a positive code into status[b] (int32, device, one per sequence).
@@ -90,8 +89,8 @@ typedef struct {
 
 /* ---- context ------------------------------------------------------------ */
 
-/* Creates a context on a CUDA device (allocates a small device block for internal
- * flags).  confu_destroy frees it.  A context is not thread safe. */
+/* Creates a context for a CUDA device (host state only: the SM count, the workspace and
+ * paging settings, the last CUDA error).  confu_destroy frees it.  A context is not thread safe. */
 int confu_create(confu_ctx** ctx, int device);
 int confu_destroy(confu_ctx* ctx);
 

@@ -58,14 +58,11 @@ int confu_create(confu_ctx** out, int device)
     c->device = device;
     c->workspace = nullptr;
     c->workspace_bytes = 0;
-    c->dev_flags = nullptr;
     c->block_table = nullptr;
     c->max_pages = 0;
     c->last_error = cudaSuccess;
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
-    if (e == cudaSuccess) e = cudaMalloc((void**)&c->dev_flags, 256);
-    if (e == cudaSuccess) e = cudaMemset(c->dev_flags, 0, 256);
     if (e != cudaSuccess) {
         delete c;
         return CONFU_ERR_CUDA;
@@ -77,7 +74,6 @@ int confu_create(confu_ctx** out, int device)
 int confu_destroy(confu_ctx* ctx)
 {
     if (!ctx) return CONFU_ERR_ARG;
-    if (ctx->dev_flags) cudaFree(ctx->dev_flags);
     delete ctx;
     return CONFU_OK;
 }

@@ -98,7 +98,6 @@ struct Ctx {
     size_t workspace_bytes;
     const int32_t* block_table;    // paged pools when set (confu_set_paging)
     int32_t max_pages;
-    int32_t* dev_flags;        // small device block owned by the context
     cudaError_t last_error;
 };
 
