@@ -440,6 +440,89 @@ int confu_ref_tree_accept(int32_t B, int32_t T, int32_t C, int32_t V, int32_t lo
 }
 
 /* ------------------------------------------------------------------ */
+/* acceptance, sample-and-match rule                                   */
+/* ------------------------------------------------------------------ */
+static int match_one(int T, int C, int V, int dtype, const void* tl, int64_t row0,
+                     const int32_t* tokens, const int32_t* parent, const int32_t* owner,
+                     const double* uni, double temperature,
+                     int32_t* accept_len, int32_t* path, int32_t* next_token, int32_t* future_row,
+                     int32_t* counters, double* draw_margin, int32_t* alt_token)
+{
+    int32_t cnt[4] = {0, 0, 0, 0};
+    double margin = INFINITY;
+    int32_t alt[2] = {-1, -1};
+    int cur = 0, len = 0;
+    double* p = NULL;
+
+    null_outputs(accept_len, path, next_token, future_row);
+    int st = check_tree(parent, owner, T, C);
+    if (!st)
+        for (int i = 0; i < T; ++i)
+            if (tokens[i] < 0 || tokens[i] >= V) { st = CONFU_REF_ST_BAD_TOKEN; break; }
+    if (st) goto done;
+
+    if (temperature > 0.0) p = (double*)malloc((size_t)V * sizeof(double));
+    for (;;) {
+        /* the token the target model itself emits after node cur */
+        int x;
+        if (temperature > 0.0) {
+            if (!softmax_row(tl, dtype, row0 + cur, V, temperature, p)) { st = CONFU_REF_ST_NONFINITE; break; }
+            double mg;
+            x = inverse_cdf(p, V, uni[cur], &mg, alt);
+            if (mg < margin) margin = mg;
+            if (mg < 1e-5) ++cnt[2];
+        } else {
+            x = argmax_row(tl, dtype, row0 + cur, V);
+            if (x < 0) { st = CONFU_REF_ST_NONFINITE; break; }
+        }
+        ++cnt[0];
+        /* the draft token that matches it, if any (lowest node index) */
+        int hit = -1;
+        for (int c = cur + 1; c < T; ++c)
+            if (parent[c] == cur && tokens[c] == x) { hit = c; break; }
+        if (hit < 0) { *next_token = x; break; }
+        if (len + 1 > CONFU_REF_MAX_DEPTH) { st = CONFU_REF_ST_TOO_DEEP; break; }
+        path[++len] = hit;
+        cur = hit;
+        ++cnt[1];
+    }
+    free(p);
+    if (st) { null_outputs(accept_len, path, next_token, future_row); goto done; }
+    *accept_len = len;
+    if (future_row) *future_row = future_row_of(parent, owner, T, C, cur);
+
+done:
+    if (counters) memcpy(counters, cnt, sizeof cnt);
+    if (draw_margin) *draw_margin = margin;
+    if (alt_token) { alt_token[0] = alt[0]; alt_token[1] = alt[1]; }
+    return st;
+}
+
+int confu_ref_tree_accept_match(int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
+                                const void* tl, const int32_t* tokens, const int32_t* parent,
+                                const int32_t* owner, const double* uniforms, double temperature,
+                                int32_t* accept_len, int32_t* path, int32_t* next_token,
+                                int32_t* future_row, int32_t* counters, double* draw_margin,
+                                int32_t* alt_token, int32_t* status)
+{
+    if (B < 0 || T <= 0 || C < 0 || V <= 0) return -1;
+    if (logit_dtype < CONFU_REF_BF16 || logit_dtype > CONFU_REF_F64) return -1;
+    if (!tl || !tokens || !parent || !accept_len || !path || !next_token) return -1;
+    if (temperature > 0.0 && !uniforms) return -1;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        int st = match_one(T, C, V, logit_dtype, tl, (int64_t)b * T, tokens + (int64_t)b * T,
+                           parent + (int64_t)b * T, owner ? owner + (int64_t)b * C : NULL,
+                           uniforms ? uniforms + (int64_t)b * T : NULL, temperature,
+                           accept_len + b, path + (int64_t)b * (CONFU_REF_MAX_DEPTH + 1), next_token + b,
+                           future_row ? future_row + b : NULL, counters ? counters + 4 * (int64_t)b : NULL,
+                           draw_margin ? draw_margin + b : NULL, alt_token ? alt_token + 2 * (int64_t)b : NULL);
+        if (status) status[b] = st;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
 /* compaction                                                          */
 /* ------------------------------------------------------------------ */
 int confu_ref_kv_compact(int32_t B, int32_t n_layers, int64_t row_bytes,

@@ -118,6 +118,29 @@ int confu_ref_tree_accept(int32_t B, int32_t T, int32_t C, int32_t V, int32_t lo
                           int32_t* status);
 
 /*
+ * Acceptance by the sample-and-match rule, Sec. 2 steps 3-4 read literally: at the
+ * current node (the root first) the target model's own next token x is drawn from
+ * softmax(target_logits[node] / temperature) by inverse CDF in index order with
+ * uniforms[b][node] (temperature 0: x = the lowest index of the largest logit); the
+ * child of the node that carries x (lowest node index) is accepted and becomes the
+ * current node; when no child carries x -- always so at a leaf -- the walk stops and
+ * x itself is the next token (the replacement of the first rejected draft, or the
+ * bonus token).  Only the target rows of the walked path are read: a non-finite
+ * logit is an error only there.  No draft logits.
+ * Outputs as for confu_ref_tree_accept, with counters [4] = {draws, accepted nodes,
+ * draws within 1e-5 of a CDF edge, 0}, draw_margin = the smallest distance of a
+ * uniform to an edge of its chosen CDF cell over all draws (+inf at temperature 0),
+ * alt_token [2] = previous / next index of non-zero weight around the LAST draw.
+ */
+int confu_ref_tree_accept_match(int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
+                                const void* target_logits, const int32_t* tokens,
+                                const int32_t* parent, const int32_t* con_owner,
+                                const double* uniforms, double temperature,
+                                int32_t* accept_len, int32_t* path, int32_t* next_token,
+                                int32_t* future_row, int32_t* counters, double* draw_margin,
+                                int32_t* alt_token, int32_t* status);
+
+/*
  * KV compaction of the accepted path ("the final accepted sequence becomes the
  * input for the next drafting step", Sec. 2 step 4).  For every layer and for K
  * and V: new[P_b + k] = old[P_b + path[b][k]], k = 1..accept_len[b], where "old"

@@ -37,7 +37,7 @@ def lib():
         _lib = C.CDLL(_build.build())
         _lib.confu_ref_num_threads.restype = C.c_int
         for name in ("confu_ref_tree_attention", "confu_ref_tree_attention_rows",
-                     "confu_ref_tree_accept", "confu_ref_kv_compact"):
+                     "confu_ref_tree_accept", "confu_ref_tree_accept_match", "confu_ref_kv_compact"):
             getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -144,6 +144,34 @@ def tree_accept(target_logits, draft_logits, tokens, parent, con_owner, uniforms
                                      _p(o["resample_margin"]), _p(o["alt_token"]), _p(o["status"]))
     if rc != 0:
         raise ValueError("confu_ref_tree_accept: bad argument")
+    return o
+
+
+def tree_accept_match(target_logits, tokens, parent, con_owner, uniforms, temperature=1.0):
+    """Acceptance by the sample-and-match rule.  Returns a dict of CPU tensors (see confu_ref.h)."""
+    B, T, V = target_logits.shape
+    Cn = 0 if con_owner is None else con_owner.shape[1]
+    tl = target_logits.contiguous()
+    tokens, parent, con_owner = _i32(tokens), _i32(parent), _i32(con_owner)
+    uni = None if uniforms is None else uniforms.to(torch.float64).contiguous()
+    o = {
+        "accept_len": torch.zeros(B, dtype=torch.int32),
+        "path": torch.full((B, MAX_DEPTH + 1), -1, dtype=torch.int32),
+        "next_token": torch.zeros(B, dtype=torch.int32),
+        "future_row": torch.zeros(B, dtype=torch.int32),
+        "counters": torch.zeros(B, 4, dtype=torch.int32),
+        "draw_margin": torch.zeros(B, dtype=torch.float64),
+        "alt_token": torch.zeros(B, 2, dtype=torch.int32),
+        "status": torch.zeros(B, dtype=torch.int32),
+    }
+    rc = lib().confu_ref_tree_accept_match(C.c_int32(B), C.c_int32(T), C.c_int32(Cn), C.c_int32(V),
+                                           C.c_int32(_DT[tl.dtype]), _p(tl), _p(tokens), _p(parent),
+                                           _p(con_owner), _p(uni), C.c_double(temperature),
+                                           _p(o["accept_len"]), _p(o["path"]), _p(o["next_token"]),
+                                           _p(o["future_row"]), _p(o["counters"]), _p(o["draw_margin"]),
+                                           _p(o["alt_token"]), _p(o["status"]))
+    if rc != 0:
+        raise ValueError("confu_ref_tree_accept_match: bad argument")
     return o
 
 
