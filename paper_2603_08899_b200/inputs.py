@@ -231,7 +231,7 @@ def draft_tokens(cfg: VerifyConfig, parent: torch.Tensor, draft_logits: torch.Te
             row = draft_logits[b, u].float()
             if temperature > 0:
                 uu = torch.rand(row.shape, generator=g, device=device, dtype=torch.float32)
-                gumbel = -torch.log(-torch.log(uu.clamp_min(1e-20)).clamp_min(1e-20))
+                gumbel = -torch.log((-torch.log(uu.clamp_min(1e-20))).clamp_min(1e-20))
                 row = row / temperature + gumbel
             top = torch.topk(row, len(ch)).indices.cpu()
             for c, t in zip(ch, top.tolist()):
