@@ -214,6 +214,27 @@ int confu_tree_accept_static(int32_t B, int32_t T, int32_t C, int32_t V, int32_t
                              int32_t* accept_len, int32_t* path, int32_t* next_token, int32_t* future_row,
                              int32_t* counters, int32_t* status, void* stream);
 
+/*
+ * Acceptance by the sample-and-match rule (Sec. 2 steps 3-4 as the text states them: a draft
+ * token is accepted if it matches the token sampled from the target model's distribution at its
+ * position; the first mismatch is replaced by the target's own token).  Walk from the root: at the
+ * current node draw x from softmax(target_logits[node] / temperature) by inverse CDF in index
+ * order with uniforms[b][node] (temperature 0: x = lowest index of the largest logit); the child
+ * that carries x (lowest node index) is accepted and becomes the current node; if none does --
+ * always so at a leaf -- the walk ends and next_token = x.  Every emitted token is a sample of
+ * the target model, so the output distribution is the target's.
+ * Statistics are computed on demand: only the target rows of the walked path are read
+ * ((accept_len + 1) * V logits per sequence) and a non-finite logit is an error (status 5) only
+ * there.  No draft logits, no workspace.
+ * Outputs as for confu_tree_accept; counters (optional) [B][4] = draws, accepted nodes,
+ * reserved, reserved.  All pointers device.
+ */
+int confu_tree_accept_match(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
+                            const void* target_logits, const int32_t* tokens, const int32_t* parent,
+                            const int32_t* con_owner, const float* uniforms, float temperature,
+                            int32_t* accept_len, int32_t* path, int32_t* next_token, int32_t* future_row,
+                            int32_t* counters, int32_t* status, void* stream);
+
 /* ---- KV compaction (Sec. 2 step 4: the accepted sequence is the next input) ---- */
 
 /*

@@ -23,6 +23,7 @@ EXPORTS = [
     "confu_last_cuda_error", "confu_plan_bytes", "confu_tree_plan", "confu_tree_attention",
     "confu_accept_workspace_bytes", "confu_tree_accept", "confu_kv_compact", "confu_kv_append",
     "confu_tree_accept_static_max_rows", "confu_tree_accept_static", "confu_set_paging",
+    "confu_tree_accept_match",
 ]
 
 
@@ -49,7 +50,8 @@ def lib():
         L.confu_status_string.restype = C.c_char_p
         L.confu_last_cuda_error.restype = C.c_char_p
         for n in ("confu_create", "confu_destroy", "confu_set_workspace", "confu_tree_plan", "confu_tree_attention",
-                  "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static", "confu_set_paging"):
+                  "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static", "confu_set_paging",
+                  "confu_tree_accept_match"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -149,6 +151,17 @@ def confu_tree_accept(ctx, B, T, Cn, V, logit_dtype, target_logits, draft_logits
                                    C.c_float(temperature), C.c_int32(sibling_mode), _ptr(accept_len), _ptr(path),
                                    _ptr(next_token), _ptr(future_row), _ptr(counters), _ptr(workspace),
                                    C.c_size_t(ws_bytes), _ptr(status), _stream(stream)), ctx)
+
+
+def confu_tree_accept_match(ctx, B, T, Cn, V, logit_dtype, target_logits, tokens, parent, con_owner, uniforms,
+                            temperature, accept_len, path, next_token, future_row, counters, status, stream=None):
+    """Acceptance by the sample-and-match rule; reads only the target rows of the walked path."""
+    _check("confu_tree_accept_match",
+           lib().confu_tree_accept_match(ctx, C.c_int32(B), C.c_int32(T), C.c_int32(Cn), C.c_int32(V),
+                                         C.c_int32(dtype_code(logit_dtype)), _ptr(target_logits), _ptr(tokens),
+                                         _ptr(parent), _ptr(con_owner), _ptr(uniforms), C.c_float(temperature),
+                                         _ptr(accept_len), _ptr(path), _ptr(next_token), _ptr(future_row),
+                                         _ptr(counters), _ptr(status), _stream(stream)), ctx)
 
 
 def confu_tree_accept_static_max_rows():

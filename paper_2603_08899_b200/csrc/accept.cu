@@ -11,6 +11,9 @@
 //                      the cluster runs the same control flow on the same data; only the passes over
 //                      the vocabulary are shared out (strip s to CTA s mod kWalkCluster), the strip
 //                      sums being written into every CTA's shared memory before a cluster barrier.
+//   match_walk_kernel  the sample-and-match rule, same cluster layout, no statistics kernel: at each
+//                      node of the walked path the row's maximum, its softmax weights and the
+//                      inverse CDF are computed on the spot, so only those rows are ever read.
 #include <cooperative_groups.h>
 #include <limits.h>
 
@@ -206,6 +209,10 @@ struct WalkShared {
     int tests, rejections;
     int strip_sel;
     double strip_off, target;
+    // row maximum of match_walk_kernel: per warp, then per CTA of the cluster
+    float red_m[kWalkThreads / 32], cl_m[kWalkCluster];
+    int red_arg[kWalkThreads / 32], red_flag[kWalkThreads / 32], cl_arg[kWalkCluster], cl_flag[kWalkCluster];
+    int next;
 };
 
 // merged statistics of one row from its chunk partials (fixed order)
@@ -544,6 +551,191 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
             counters[4 * b + 2] = 0; counters[4 * b + 3] = 0;
         }
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// K4b: sample-and-match walk with statistics on demand
+// ---------------------------------------------------------------------------------------------
+// Largest logit of a row, its lowest index and a non-finite flag; every CTA of the cluster gets
+// the same three values (strips shared out as in full_pass, partial results exchanged through
+// distributed shared memory and merged in rank order).
+template <typename T>
+__device__ void max_pass(const T* __restrict__ trow, int V, bool vec_ok, WalkShared& sh, float& M, int& arg, int& flag)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int tid = threadIdx.x, n_strips = (V + kStrip - 1) / kStrip;
+    float m = -INFINITY;
+    int a = INT_MAX, f = 0;
+    for (int st = rank; st < n_strips; st += kWalkCluster) {
+        const int i0 = st * kStrip + tid * kEpt;
+        float x[kEpt];
+        load8(trow, i0, V, vec_ok, x);
+#pragma unroll
+        for (int j = 0; j < kEpt; ++j) {
+            if (i0 + j < V) {
+                if (!(fabsf(x[j]) <= 3.0e38f)) f = 1;
+                if (x[j] > m) { m = x[j]; a = i0 + j; }
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, o);
+        const int oa = __shfl_xor_sync(0xffffffffu, a, o);
+        f |= __shfl_xor_sync(0xffffffffu, f, o);
+        if (om > m || (om == m && oa < a)) { m = om; a = oa; }
+    }
+    if ((tid & 31) == 0) { sh.red_m[tid >> 5] = m; sh.red_arg[tid >> 5] = a; sh.red_flag[tid >> 5] = f; }
+    __syncthreads();
+    // every CTA has finished reading the previous exchange: it may be overwritten
+    cluster.sync();
+    if (tid < kWalkCluster) {
+        float bm = -INFINITY;
+        int ba = INT_MAX, bf = 0;
+        for (int w = 0; w < kWalkThreads / 32; ++w) {
+            bf |= sh.red_flag[w];
+            if (sh.red_m[w] > bm || (sh.red_m[w] == bm && sh.red_arg[w] < ba)) { bm = sh.red_m[w]; ba = sh.red_arg[w]; }
+        }
+        *cluster.map_shared_rank(&sh.cl_m[rank], tid) = bm;
+        *cluster.map_shared_rank(&sh.cl_arg[rank], tid) = ba;
+        *cluster.map_shared_rank(&sh.cl_flag[rank], tid) = bf;
+    }
+    cluster.sync();
+    M = -INFINITY; arg = INT_MAX; flag = 0;
+    for (int r = 0; r < kWalkCluster; ++r) {
+        flag |= sh.cl_flag[r];
+        if (sh.cl_m[r] > M || (sh.cl_m[r] == M && sh.cl_arg[r] < arg)) { M = sh.cl_m[r]; arg = sh.cl_arg[r]; }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kWalkThreads) match_walk_kernel(
+    int Tn, int C, int V, const T* __restrict__ tl, const int32_t* __restrict__ tokens,
+    const int32_t* __restrict__ parent, const int32_t* __restrict__ con_owner, const float* __restrict__ uniforms,
+    float temperature, int32_t* __restrict__ accept_len, int32_t* __restrict__ path, int32_t* __restrict__ next_token,
+    int32_t* __restrict__ future_row, int32_t* __restrict__ counters, int32_t* __restrict__ status)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    WalkShared& sh = *reinterpret_cast<WalkShared*>(smem_raw);
+    const int b = blockIdx.x / kWalkCluster, tid = threadIdx.x;
+    const bool writer = blockIdx.x % kWalkCluster == 0;
+    const int32_t* par = parent + (size_t)b * Tn;
+    const int32_t* tok = tokens + (size_t)b * Tn;
+    const int32_t* own = con_owner ? con_owner + (size_t)b * C : nullptr;
+    const bool greedy = !(temperature > 0.f);
+    const bool vec_ok = ((size_t)V * sizeof(T)) % 16 == 0;
+    const float k2 = (greedy ? 1.f : 1.f / temperature) * kLog2e;
+    int32_t* pth = path + (size_t)b * kPathLen;
+
+    if (tid == 0) { sh.code = INT_MAX; sh.cur = 0; sh.len = 0; sh.path[0] = 0; sh.tests = 0; sh.accepted = 0; sh.done = 0; sh.next = -1; }
+    __syncthreads();
+    if (tid < Tn) {
+        const int p = par[tid];
+        if (tid == 0 ? (p != -1) : (p < 0 || p >= tid)) atomicMin(&sh.code, (int)CONFU_ST_BAD_PARENT);
+        else if (tok[tid] < 0 || tok[tid] >= V) atomicMin(&sh.code, (int)CONFU_ST_BAD_TOKEN);
+    }
+    if (tid < C) {
+        const int o = own[tid];
+        if (o < 0 || o >= Tn) atomicMin(&sh.code, (int)CONFU_ST_BAD_OWNER);
+    }
+    __syncthreads();
+    int code = sh.code == INT_MAX ? 0 : sh.code;
+    while (!code) {
+        const int cur = sh.cur;
+        const T* trow = tl + ((size_t)b * Tn + cur) * V;
+        float M;
+        int arg, flag;
+        max_pass(trow, V, vec_ok, sh, M, arg, flag);
+        if (flag) { code = CONFU_ST_NONFINITE; break; }
+        int x = arg;
+        if (!greedy) {
+            // weights 2^((x - M) k2), unnormalised: the inverse CDF scales the uniform by their sum
+            if (tid == 0) { sh.Mt = M; sh.invZt = 1.f; }
+            __syncthreads();
+            full_pass(trow, trow, V, vec_ok, 0, 0, sh, k2);
+            x = locate(trow, trow, V, vec_ok, 0, 0, sh, k2, (double)uniforms[(size_t)b * Tn + cur]);
+        }
+        if (tid == 0) {
+            ++sh.tests;
+            int hit = -1;
+            for (int c = cur + 1; c < Tn; ++c)
+                if (par[c] == cur && tok[c] == x) { hit = c; break; }
+            if (hit < 0) { sh.next = x; sh.done = 1; }
+            else if (sh.len + 1 > CONFU_MAX_DEPTH) sh.done = 3;
+            else { sh.path[++sh.len] = hit; sh.cur = hit; ++sh.accepted; }
+        }
+        __syncthreads();
+        if (sh.done == 3) code = CONFU_ST_TOO_DEEP;
+        if (sh.done) break;
+    }
+    if (code) {
+        if (writer && tid < kPathLen) pth[tid] = tid == 0 ? 0 : -1;
+        if (writer && tid == 0) {
+            accept_len[b] = 0; next_token[b] = -1;
+            if (future_row) future_row[b] = -1;
+            if (counters) { counters[4 * b] = 0; counters[4 * b + 1] = 0; counters[4 * b + 2] = 0; counters[4 * b + 3] = 0; }
+            if (status) status[b] = code;
+        }
+        return;
+    }
+    if (writer && tid < kPathLen) pth[tid] = tid <= sh.len ? sh.path[tid] : -1;
+    if (writer && tid == 0) {
+        accept_len[b] = sh.len;
+        next_token[b] = sh.next;
+        if (future_row) {
+            int fr = -1;
+            for (int a = sh.cur; a >= 0 && fr < 0; a = par[a])
+                for (int k = 0; k < C; ++k)
+                    if (own[k] == a) { fr = Tn + k; break; }
+            future_row[b] = fr;
+        }
+        if (counters) { counters[4 * b] = sh.tests; counters[4 * b + 1] = sh.accepted; counters[4 * b + 2] = 0; counters[4 * b + 3] = 0; }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_match_t(int B, int Tn, int C, int V, const void* tl, const int32_t* tokens,
+                                  const int32_t* parent, const int32_t* con_owner, const float* uniforms,
+                                  float temperature, int32_t* accept_len, int32_t* path, int32_t* next_token,
+                                  int32_t* future_row, int32_t* counters, int32_t* status, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    const size_t smem = sizeof(WalkShared);
+    static bool attr_done[2] = {false, false};
+    const int ti = sizeof(T) == 2 ? 0 : 1;
+    if (!attr_done[ti]) {
+        cudaError_t e = cudaFuncSetAttribute(match_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done[ti] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)B * kWalkCluster);
+    cfg.blockDim = dim3(kWalkThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kWalkCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, match_walk_kernel<T>, Tn, C, V, (const T*)tl, tokens, parent, con_owner, uniforms,
+                              temperature, accept_len, path, next_token, future_row, counters, status);
+}
+
+cudaError_t launch_accept_match(int B, int T, int C, int V, int logit_dtype, const void* tl, const int32_t* tokens,
+                                const int32_t* parent, const int32_t* con_owner, const float* uniforms,
+                                float temperature, int32_t* accept_len, int32_t* path, int32_t* next_token,
+                                int32_t* future_row, int32_t* counters, int32_t* status, cudaStream_t st)
+{
+    if (logit_dtype == CONFU_F32)
+        return launch_match_t<float>(B, T, C, V, tl, tokens, parent, con_owner, uniforms, temperature, accept_len, path,
+                                     next_token, future_row, counters, status, st);
+    return launch_match_t<__nv_bfloat16>(B, T, C, V, tl, tokens, parent, con_owner, uniforms, temperature, accept_len,
+                                         path, next_token, future_row, counters, status, st);
 }
 
 template <typename T>

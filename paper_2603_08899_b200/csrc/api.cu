@@ -217,6 +217,28 @@ int confu_tree_accept(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
 }
 
+int confu_tree_accept_match(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
+                            const void* target_logits, const int32_t* tokens, const int32_t* parent,
+                            const int32_t* con_owner, const float* uniforms, float temperature, int32_t* accept_len,
+                            int32_t* path, int32_t* next_token, int32_t* future_row, int32_t* counters, int32_t* status,
+                            void* stream)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    if (B < 0 || T <= 0 || C < 0 || V <= 0) return CONFU_ERR_SHAPE;
+    if (logit_dtype != CONFU_BF16 && logit_dtype != CONFU_F32) return CONFU_ERR_ARG;
+    if (!(temperature >= 0.f)) return CONFU_ERR_ARG;
+    if (T > CONFU_MAX_TREE || C > CONFU_MAX_TREE || V > 262144) return CONFU_ERR_UNSUPPORTED;
+    if (B == 0) return CONFU_OK;
+    if (!target_logits || !tokens || !parent || !accept_len || !path || !next_token) return CONFU_ERR_ARG;
+    if (C > 0 && !con_owner) return CONFU_ERR_ARG;
+    if (temperature > 0.f && !uniforms) return CONFU_ERR_ARG;
+    if (misaligned(target_logits)) return CONFU_ERR_ALIGN;
+    cudaError_t e = launch_accept_match(B, T, C, V, logit_dtype, target_logits, tokens, parent, con_owner, uniforms,
+                                        temperature, accept_len, path, next_token, future_row, counters, status,
+                                        (cudaStream_t)stream);
+    return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
+}
+
 int confu_kv_compact(confu_ctx* ctx, const confu_dims* dims, int32_t n_layers, void* const* k_cache_layers,
                      void* const* v_cache_layers, const int64_t* seq_start, const int32_t* prefix_len,
                      const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len, int32_t* status,

@@ -180,6 +180,11 @@ cudaError_t launch_accept(const Ctx* ctx, int B, int T, int C, int V, int logit_
                           void* workspace, int32_t* status, cudaStream_t st);
 size_t accept_workspace_bytes(int B, int T, int V);
 
+cudaError_t launch_accept_match(int B, int T, int C, int V, int logit_dtype, const void* tl, const int32_t* tokens,
+                                const int32_t* parent, const int32_t* con_owner, const float* uniforms,
+                                float temperature, int32_t* accept_len, int32_t* path, int32_t* next_token,
+                                int32_t* future_row, int32_t* counters, int32_t* status, cudaStream_t st);
+
 cudaError_t launch_compact(const Ctx* ctx, int B, int n_layers, int64_t row_bytes, void* const* k_layers,
                            void* const* v_layers, const SlotMap& map, const int32_t* prefix_len,
                            const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len,
