@@ -76,6 +76,7 @@ enum { CONFU_BF16 = 0, CONFU_F32 = 1 };
 #define CONFU_MAX_TREE  64      /* T: tree rows (one 64-bit ancestor word per row) */
 #define CONFU_MAX_ROWS  128     /* R = T + C, with C <= 64: covers one contemplate row per node (R = 2T) */
 #define CONFU_MAX_DEPTH 63      /* path buffers hold CONFU_MAX_DEPTH + 1 node ids */
+#define CONFU_ACCEPT_LAZY 0x100 /* or-ed into sibling_mode: row statistics on demand (see confu_tree_accept) */
 
 typedef struct {
     int32_t B;          /* sequences */
@@ -182,6 +183,12 @@ size_t confu_accept_workspace_bytes(int32_t B, int32_t T, int32_t V);
  * accepted node, else by its nearest ancestor that has one, else -1; counters
  * (optional) [B][4] = ratio tests, rejections, reserved, reserved.
  * workspace: confu_accept_workspace_bytes().  All pointers device.
+ * By default one streaming pass takes the softmax statistics of all T rows of both matrices
+ * first, and a non-finite logit anywhere in them is an error (status 5).  With
+ * sibling_mode | CONFU_ACCEPT_LAZY the statistics of a row are computed when the walk reaches its
+ * node: only the rows of the walked path are read (two per visited node; greedy: the target row
+ * of every node whose children are compared), a non-finite logit is an error only there, and the
+ * workspace is not used (it may be NULL).  Decisions are the same up to rounding of the normalisers.
  */
 int confu_tree_accept(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
                       const void* target_logits, const void* draft_logits,

@@ -297,6 +297,9 @@ static int accept_one(int T, int C, int V, int dtype,
     int32_t alt[2] = {-1, -1};
     int st = CONFU_REF_ST_OK;
     int cur = 0, len = 0;
+    /* statistics on demand: only the rows the walk needs are looked at (and checked) */
+    const int lazy = (sibling_mode & CONFU_REF_ACCEPT_LAZY) != 0;
+    sibling_mode &= ~CONFU_REF_ACCEPT_LAZY;
 
     null_outputs(accept_len, path, next_token, future_row);
 
@@ -308,7 +311,7 @@ static int accept_one(int T, int C, int V, int dtype,
         for (int i = 1; i < T && !st; ++i)
             for (int j = i + 1; j < T; ++j)
                 if (parent[i] == parent[j] && tokens[i] == tokens[j]) { st = CONFU_REF_ST_DUP_SIBLING; break; }
-    if (!st) {
+    if (!st && !lazy) {
         /* a non-finite logit anywhere in the rows the step is defined on is an input error */
         for (int i = 0; i < T && !st; ++i)
             for (int v = 0; v < V; ++v) {
@@ -334,21 +337,28 @@ static int accept_one(int T, int C, int V, int dtype,
             depth[i] = depth[pa] + 1;
             if (!keep[pa]) continue;
             if (amax[pa] == -2) amax[pa] = argmax_row(tl, dtype, row0 + pa, V);
+            if (amax[pa] == -1) { st = CONFU_REF_ST_NONFINITE; break; }
             keep[i] = (tokens[i] == amax[pa]);
             if (keep[i] && depth[i] > depth[best]) best = i;
         }
         len = depth[best];
-        if (len > CONFU_REF_MAX_DEPTH) { st = CONFU_REF_ST_TOO_DEEP; free(keep); free(depth); free(amax); goto done; }
-        for (int a = best, k = len; a >= 0; a = parent[a], --k) path[k] = a;
-        cur = best;
-        *next_token = argmax_row(tl, dtype, row0 + cur, V);
+        if (!st && len > CONFU_REF_MAX_DEPTH) st = CONFU_REF_ST_TOO_DEEP;
+        if (!st) {
+            for (int a = best, k = len; a >= 0; a = parent[a], --k) path[k] = a;
+            cur = best;
+            *next_token = argmax_row(tl, dtype, row0 + cur, V);
+            if (*next_token < 0) st = CONFU_REF_ST_NONFINITE;
+        }
         free(keep); free(depth); free(amax);
+        if (st) { null_outputs(accept_len, path, next_token, future_row); goto done; }
     } else {
         double* p = (double*)malloc((size_t)V * sizeof(double));
         double* qd = (double*)malloc((size_t)V * sizeof(double));
         double* p_cur = (double*)malloc((size_t)V * sizeof(double));
         for (;;) {
-            softmax_row(tl, dtype, row0 + cur, V, temperature, p_cur);
+            /* (with the check of all rows up front these two cannot fail) */
+            if (!softmax_row(dl, dtype, row0 + cur, V, temperature, qd) ||
+                !softmax_row(tl, dtype, row0 + cur, V, temperature, p_cur)) { st = CONFU_REF_ST_NONFINITE; break; }
             /* children of cur in increasing node index */
             int n_child = 0;
             for (int i = cur + 1; i < T; ++i) if (parent[i] == cur) ++n_child;
@@ -357,7 +367,6 @@ static int accept_one(int T, int C, int V, int dtype,
                 break;
             }
             memcpy(p, p_cur, (size_t)V * sizeof(double));
-            softmax_row(dl, dtype, row0 + cur, V, temperature, qd);
             int accepted = -1, q_alive = 1;
             for (int c = cur + 1; c < T && q_alive; ++c) {
                 if (parent[c] != cur) continue;
@@ -395,7 +404,11 @@ static int accept_one(int T, int C, int V, int dtype,
             break;
         }
         free(p); free(qd); free(p_cur);
-        if (st == CONFU_REF_ST_TOO_DEEP) { null_outputs(accept_len, path, next_token, future_row); goto done; }
+        if (st == CONFU_REF_ST_TOO_DEEP || st == CONFU_REF_ST_NONFINITE) {      /* an error leaves no partial result */
+            null_outputs(accept_len, path, next_token, future_row);
+            memset(cnt, 0, sizeof cnt);
+            goto done;
+        }
         if (smargin < 1e-5) ++cnt[3];
     }
     *accept_len = len;
@@ -487,7 +500,7 @@ static int match_one(int T, int C, int V, int dtype, const void* tl, int64_t row
         ++cnt[1];
     }
     free(p);
-    if (st) { null_outputs(accept_len, path, next_token, future_row); goto done; }
+    if (st) { null_outputs(accept_len, path, next_token, future_row); memset(cnt, 0, sizeof cnt); goto done; }
     *accept_len = len;
     if (future_row) *future_row = future_row_of(parent, owner, T, C, cur);
 

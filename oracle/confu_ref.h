@@ -44,6 +44,7 @@ enum {
 };
 
 #define CONFU_REF_MAX_DEPTH 63     /* path holds CONFU_REF_MAX_DEPTH + 1 node ids */
+#define CONFU_REF_ACCEPT_LAZY 0x100
 
 typedef struct {
     int32_t B, Hq, Hkv, D, T, C, S;
@@ -98,7 +99,11 @@ int confu_ref_tree_attention_rows(const confu_ref_dims* dims,
  * node i, slot 0 the final resample / bonus draw.
  * temperature 0 -> greedy.  sibling_mode 1: children drawn without replacement
  * (after a rejection the rejected token is removed from q and q renormalised);
- * 0: children i.i.d. (q unchanged).
+ * 0: children i.i.d. (q unchanged).  A non-finite logit anywhere in the T rows
+ * (target; draft too unless greedy) is an error -- unless CONFU_REF_ACCEPT_LAZY is
+ * or-ed into sibling_mode: then only the rows the walk needs are looked at (both
+ * rows of every visited node; greedy: the target row of every node whose children
+ * are compared, and of the last node) and only they can raise that error.
  * Outputs per sequence: accept_len, path [CONFU_REF_MAX_DEPTH+1] (root first, -1
  * padded), next_token, future_row (in [T,T+C) or -1), counters [4] = {ratio
  * tests, rejections, ratio tests with |ratio-u| < 1e-5, resample draws within

@@ -212,6 +212,8 @@ struct WalkShared {
     // row maximum of match_walk_kernel: per warp, then per CTA of the cluster
     float red_m[kWalkThreads / 32], cl_m[kWalkCluster];
     int red_arg[kWalkThreads / 32], red_flag[kWalkThreads / 32], cl_arg[kWalkCluster], cl_flag[kWalkCluster];
+    // maximum and sum of exponentials of two rows at once (statistics on demand)
+    float red2_m[2][kWalkThreads / 32], red2_s[2][kWalkThreads / 32], cl2_m[2][kWalkCluster], cl2_s[2][kWalkCluster];
     int next;
 };
 
@@ -360,10 +362,101 @@ __device__ int locate(const T* __restrict__ trow, const T* __restrict__ drow, in
 }
 
 template <typename T>
+__device__ void max_pass(const T* __restrict__ trow, int V, bool vec_ok, WalkShared& sh, float& M, int& arg, int& flag);
+
+// (m, s) <- merge of two (maximum, sum of 2^((x - maximum) k2)) pairs; an empty pair is (-inf, 0)
+__device__ __forceinline__ void ms_merge(float& m, float& s, float om, float os, float k2)
+{
+    const float M = fmaxf(m, om);
+    if (M == -INFINITY) { s = 0.f; return; }
+    s = s * ex2((m - M) * k2) + os * ex2((om - M) * k2);
+    m = M;
+}
+
+// Statistics on demand: maximum and sum of 2^((x - maximum) k2) of the target row and of the draft
+// row of one node in a single pass over both (online softmax per thread, merged per warp, per CTA
+// and over the cluster in a fixed order); flag: a non-finite logit in either row.
+template <typename T>
+__device__ void stats_pass(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok, WalkShared& sh,
+                           float k2, float (&M)[2], double (&Z)[2], int& flag)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int tid = threadIdx.x, n_strips = (V + kStrip - 1) / kStrip;
+    float m[2] = {-INFINITY, -INFINITY}, s[2] = {0.f, 0.f};
+    int f = 0;
+    for (int st = rank; st < n_strips; st += kWalkCluster) {
+        const int i0 = st * kStrip + tid * kEpt;
+        float x[2][kEpt];
+        load8(trow, i0, V, vec_ok, x[0]);
+        load8(drow, i0, V, vec_ok, x[1]);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            float vm = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < kEpt; ++j) {
+                if (i0 + j < V) {
+                    if (!(fabsf(x[r][j]) <= 3.0e38f)) f = 1;
+                    vm = fmaxf(vm, x[r][j]);
+                }
+            }
+            if (vm > m[r]) { s[r] *= ex2((m[r] - vm) * k2); m[r] = vm; }
+            if (m[r] > -INFINITY) {
+#pragma unroll
+                for (int j = 0; j < kEpt; ++j) s[r] += ex2((x[r][j] - m[r]) * k2);      // padding is -inf: weight 0
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        f |= __shfl_xor_sync(0xffffffffu, f, o);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const float om = __shfl_xor_sync(0xffffffffu, m[r], o), os = __shfl_xor_sync(0xffffffffu, s[r], o);
+            // the same operand order in both partners, so that every lane ends with the same bits
+            if ((tid & o) == 0) ms_merge(m[r], s[r], om, os, k2);
+            else { float a = om, b = os; ms_merge(a, b, m[r], s[r], k2); m[r] = a; s[r] = b; }
+        }
+    }
+    if ((tid & 31) == 0) {
+        sh.red_flag[tid >> 5] = f;
+        for (int r = 0; r < 2; ++r) { sh.red2_m[r][tid >> 5] = m[r]; sh.red2_s[r][tid >> 5] = s[r]; }
+    }
+    __syncthreads();
+    cluster.sync();                      // every CTA has finished reading the previous exchange
+    if (tid < kWalkCluster) {
+        int bf = 0;
+        float bm[2] = {-INFINITY, -INFINITY}, bs[2] = {0.f, 0.f};
+        for (int w = 0; w < kWalkThreads / 32; ++w) {
+            bf |= sh.red_flag[w];
+            for (int r = 0; r < 2; ++r) ms_merge(bm[r], bs[r], sh.red2_m[r][w], sh.red2_s[r][w], k2);
+        }
+        *cluster.map_shared_rank(&sh.cl_flag[rank], tid) = bf;
+        for (int r = 0; r < 2; ++r) {
+            *cluster.map_shared_rank(&sh.cl2_m[r][rank], tid) = bm[r];
+            *cluster.map_shared_rank(&sh.cl2_s[r][rank], tid) = bs[r];
+        }
+    }
+    cluster.sync();
+    flag = 0;
+    for (int c = 0; c < kWalkCluster; ++c) flag |= sh.cl_flag[c];
+    for (int r = 0; r < 2; ++r) {
+        float mm = -INFINITY;
+        for (int c = 0; c < kWalkCluster; ++c) mm = fmaxf(mm, sh.cl2_m[r][c]);
+        double z = 0.0;
+        for (int c = 0; c < kWalkCluster; ++c)
+            if (sh.cl2_m[r][c] > -INFINITY) z += (double)sh.cl2_s[r][c] * exp2((double)(sh.cl2_m[r][c] - mm) * (double)k2);
+        M[r] = mm;
+        Z[r] = z;
+    }
+}
+
+template <typename T>
 __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
     int Tn, int C, int V, const T* __restrict__ tl, const T* __restrict__ dl, const int32_t* __restrict__ tokens,
     const int32_t* __restrict__ parent, const int32_t* __restrict__ con_owner, const float* __restrict__ uniforms,
-    float temperature, int mode, int nch, int n_rows, const RowStat* __restrict__ stats,
+    float temperature, int mode, int lazy, int nch, int n_rows, const RowStat* __restrict__ stats,
     int32_t* __restrict__ accept_len, int32_t* __restrict__ path, int32_t* __restrict__ next_token,
     int32_t* __restrict__ future_row, int32_t* __restrict__ counters, int32_t* __restrict__ status)
 {
@@ -391,7 +484,7 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
             if (!greedy && mode == 1 && tid > 0)
                 for (int j = tid + 1; j < Tn; ++j)
                     if (par[j] == p && tok[j] == tok[tid]) code = CONFU_ST_DUP_SIBLING;
-            if (code == INT_MAX)
+            if (code == INT_MAX && !lazy)
                 for (int c = 0; c < nch; ++c)
                     if (st_t[(size_t)tid * kStatChunksMax + c].flag ||
                         (!greedy && st_d[(size_t)tid * kStatChunksMax + c].flag))
@@ -420,7 +513,52 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
 
     if (tid == 0) { sh.cur = 0; sh.len = 0; sh.path[0] = 0; sh.tests = 0; sh.rejections = 0; sh.done = 0; }
 
-    if (greedy) {
+    int lazy_code = 0;                // statistics on demand: a non-finite logit in a row that was needed
+    if (greedy && lazy) {
+        // the same walk as below, node by node, with the argmax of a row computed when the first
+        // child of a kept node comes up (every CTA of the cluster takes the same branches)
+        if (tid == 0) { sh.k = 0; sh.cur = 0; sh.len = 0; }
+        if (tid < Tn) sh.amax[tid] = -2;
+        __syncthreads();
+        unsigned long long keep = 1ull;
+        for (int i = 1; i < Tn && !lazy_code; ++i) {
+            const int pa = par[i];
+            if (!((keep >> pa) & 1ull)) continue;
+            if (sh.amax[pa] == -2) {
+                float M; int a, flag;
+                max_pass(tl + ((size_t)b * Tn + pa) * V, V, vec_ok, sh, M, a, flag);
+                if (flag) { lazy_code = CONFU_ST_NONFINITE; break; }
+                __syncthreads();
+                if (tid == 0) sh.amax[pa] = a;
+                __syncthreads();
+            }
+            if (tok[i] == sh.amax[pa]) keep |= 1ull << i;
+        }
+        if (!lazy_code) {
+            // deepest kept node, lowest index on ties; its own row gives the next token
+            int best = 0, best_depth = 0;
+            for (int i = 1; i < Tn; ++i) {
+                if (!((keep >> i) & 1ull)) continue;
+                int d = 0;
+                for (int a = i; a > 0; a = par[a]) ++d;
+                if (d > best_depth) { best = i; best_depth = d; }
+            }
+            int a_best = sh.amax[best];
+            if (a_best == -2) {
+                float M; int flag;
+                max_pass(tl + ((size_t)b * Tn + best) * V, V, vec_ok, sh, M, a_best, flag);
+                if (flag) lazy_code = CONFU_ST_NONFINITE;
+            }
+            __syncthreads();
+            if (tid == 0 && !lazy_code) {
+                sh.len = best_depth;
+                for (int a = best, k = best_depth; a >= 0; a = par[a], --k) sh.path[k] = a;
+                sh.cur = best;
+                if (writer) next_token[b] = a_best;
+            }
+            __syncthreads();
+        }
+    } else if (greedy) {
         if (tid < Tn) {
             float M; double Z; int a;
             merge_row(st_t + (size_t)tid * kStatChunksMax, nch, 1.0, M, Z, a);
@@ -451,13 +589,28 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
         const double u0 = (double)uniforms[(size_t)b * Tn];
         for (;;) {
             // ---- set up the current node ----
+            if (lazy) {
+                // maximum and normaliser of the node's two rows, computed now
+                __syncthreads();
+                const T* rt = tl + ((size_t)b * Tn + sh.cur) * V;
+                const T* rd = dl + ((size_t)b * Tn + sh.cur) * V;
+                float M[2];
+                double Z[2];
+                int flag;
+                stats_pass(rt, rd, V, vec_ok, sh, k2, M, Z, flag);
+                if (flag) { lazy_code = CONFU_ST_NONFINITE; break; }
+                __syncthreads();
+                if (tid == 0) { sh.Mt = M[0]; sh.invZt = (float)(1.0 / Z[0]); sh.Md = M[1]; sh.invZd = (float)(1.0 / Z[1]); }
+            }
             if (tid == 0) {
                 const int cur = sh.cur;
-                float M; double Z; int a;
-                merge_row(st_t + (size_t)cur * kStatChunksMax, nch, inv_temp, M, Z, a);
-                sh.Mt = M; sh.invZt = (float)(1.0 / Z);
-                merge_row(st_d + (size_t)cur * kStatChunksMax, nch, inv_temp, M, Z, a);
-                sh.Md = M; sh.invZd = (float)(1.0 / Z);
+                if (!lazy) {
+                    float M; double Z; int a;
+                    merge_row(st_t + (size_t)cur * kStatChunksMax, nch, inv_temp, M, Z, a);
+                    sh.Mt = M; sh.invZt = (float)(1.0 / Z);
+                    merge_row(st_d + (size_t)cur * kStatChunksMax, nch, inv_temp, M, Z, a);
+                    sh.Md = M; sh.invZd = (float)(1.0 / Z);
+                }
                 int n = 0;
                 for (int i = cur + 1; i < Tn; ++i) if (par[i] == cur) sh.ch[n++] = i;
                 sh.nch = n; sh.k = 0; sh.accepted = -1;
@@ -534,6 +687,16 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
             return;
         }
         if (sh.done == 2 && writer && tid == 0 && status) status[b] = CONFU_ST_DEGENERATE;
+    }
+    if (lazy_code) {
+        if (writer && tid < kPathLen) pth[tid] = tid == 0 ? 0 : -1;
+        if (writer && tid == 0) {
+            accept_len[b] = 0; next_token[b] = -1;
+            if (future_row) future_row[b] = -1;
+            if (counters) { counters[4 * b] = 0; counters[4 * b + 1] = 0; counters[4 * b + 2] = 0; counters[4 * b + 3] = 0; }
+            if (status) status[b] = lazy_code;
+        }
+        return;
     }
     // ---- outputs ----
     if (writer && tid < kPathLen) pth[tid] = tid <= sh.len ? sh.path[tid] : -1;
@@ -741,11 +904,12 @@ cudaError_t launch_accept_match(int B, int T, int C, int V, int logit_dtype, con
 template <typename T>
 static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, const void* dl, const int32_t* tokens,
                                    const int32_t* parent, const int32_t* con_owner, const float* uniforms,
-                                   float temperature, int mode, int32_t* accept_len, int32_t* path,
+                                   float temperature, int mode_flags, int32_t* accept_len, int32_t* path,
                                    int32_t* next_token, int32_t* future_row, int32_t* counters, void* workspace,
                                    int32_t* status, cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
+    const int mode = mode_flags & 0xff, lazy = (mode_flags & CONFU_ACCEPT_LAZY) ? 1 : 0;
     const bool greedy = !(temperature > 0.f);
     const int n_rows = B * Tn;
     const int nmat = greedy ? 1 : 2;
@@ -757,10 +921,13 @@ static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, 
     nch = (V + chunk_elems - 1) / chunk_elems;
     const float k2 = (greedy ? 1.f : 1.f / temperature) * kLog2e;
     RowStat* stats = (RowStat*)workspace;
-    row_stats_kernel<T><<<dim3(n_rows, nch, nmat), 256, 0, st>>>((const T*)tl, (const T*)dl, V, n_rows, nch,
-                                                                 chunk_elems, k2, stats);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (!lazy) {
+        row_stats_kernel<T><<<dim3(n_rows, nch, nmat), 256, 0, st>>>((const T*)tl, (const T*)dl, V, n_rows, nch,
+                                                                     chunk_elems, k2, stats);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     const size_t smem = sizeof(WalkShared);
     static bool attr_done[2] = {false, false};
     const int ti = sizeof(T) == 2 ? 0 : 1;
@@ -782,7 +949,7 @@ static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, accept_walk_kernel<T>, Tn, C, V, (const T*)tl, (const T*)dl, tokens, parent, con_owner,
-                              uniforms, temperature, mode, nch, n_rows, stats, accept_len, path, next_token, future_row,
+                              uniforms, temperature, mode, lazy, nch, n_rows, stats, accept_len, path, next_token, future_row,
                               counters, status);
 }
 

@@ -61,7 +61,7 @@ int confu_tree_accept_static(int32_t B, int32_t T, int32_t C, int32_t V, int32_t
 {
     if (B < 0 || T <= 0 || C < 0 || V <= 0) return CONFU_ERR_SHAPE;
     if (logit_dtype != CONFU_BF16 && logit_dtype != CONFU_F32) return CONFU_ERR_ARG;
-    if (sibling_mode != 0 && sibling_mode != 1) return CONFU_ERR_ARG;
+    if ((sibling_mode & ~CONFU_ACCEPT_LAZY) != 0 && (sibling_mode & ~CONFU_ACCEPT_LAZY) != 1) return CONFU_ERR_ARG;
     if (!(temperature >= 0.f)) return CONFU_ERR_ARG;
     if (T > CONFU_MAX_TREE || C > CONFU_MAX_TREE || V > 262144) return CONFU_ERR_UNSUPPORTED;
     // the fixed scratch holds the statistics of at most kStaticMaxRows logit rows per matrix

@@ -202,7 +202,8 @@ int confu_tree_accept(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V
     if (!ctx) return CONFU_ERR_ARG;
     if (B < 0 || T <= 0 || C < 0 || V <= 0) return CONFU_ERR_SHAPE;
     if (logit_dtype != CONFU_BF16 && logit_dtype != CONFU_F32) return CONFU_ERR_ARG;
-    if (sibling_mode != 0 && sibling_mode != 1) return CONFU_ERR_ARG;
+    const bool lazy = (sibling_mode & CONFU_ACCEPT_LAZY) != 0;
+    if ((sibling_mode & ~CONFU_ACCEPT_LAZY) != 0 && (sibling_mode & ~CONFU_ACCEPT_LAZY) != 1) return CONFU_ERR_ARG;
     if (!(temperature >= 0.f)) return CONFU_ERR_ARG;
     if (T > CONFU_MAX_TREE || C > CONFU_MAX_TREE || V > 262144) return CONFU_ERR_UNSUPPORTED;
     if (B == 0) return CONFU_OK;
@@ -210,7 +211,7 @@ int confu_tree_accept(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V
     if (C > 0 && !con_owner) return CONFU_ERR_ARG;
     if (temperature > 0.f && (!draft_logits || !uniforms)) return CONFU_ERR_ARG;
     if (misaligned(target_logits) || misaligned(draft_logits) || misaligned(workspace)) return CONFU_ERR_ALIGN;
-    if (!workspace || workspace_bytes < accept_workspace_bytes(B, T, V)) return CONFU_ERR_WORKSPACE;
+    if (!lazy && (!workspace || workspace_bytes < accept_workspace_bytes(B, T, V))) return CONFU_ERR_WORKSPACE;
     cudaError_t e = launch_accept(ctx, B, T, C, V, logit_dtype, target_logits, draft_logits, tokens, parent, con_owner,
                                   uniforms, temperature, sibling_mode, accept_len, path, next_token, future_row,
                                   counters, workspace, status, (cudaStream_t)stream);

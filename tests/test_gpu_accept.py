@@ -145,3 +145,58 @@ def test_emitted_tokens_follow_the_target_distribution_on_gpu(gpu, mode):
     first, second = _emitted(got, tok)
     p_first, p_second = _chi2_pvalues(first, second, P0, P1)
     assert p_first > 1e-4 and p_second > 1e-4, (p_first, p_second)
+
+
+# ---------------------------------------------------------------- statistics on demand
+LAZY = 0x100
+
+
+@pytest.mark.parametrize("name", ["bf16_noise", "bf16_independent", "ragged_vocab_not_multiple_of_8", "vocab_llama",
+                                  "chain_12", "star", "single_node", "small_vocab_16"])
+@pytest.mark.parametrize("temperature", [1.0, 0.7, 0.0])
+def test_lazy_statistics_match_oracle(gpu, name, temperature):
+    cfg = CASES[name]
+    got, want = _run(gpu, cfg, temperature, mode=1 | LAZY)
+    log = []
+    exact, border = H.compare_accept(got, want, log)
+    assert exact + border == cfg.B
+    assert border <= max(1, cfg.B // 8), log
+
+
+def test_lazy_statistics_need_no_workspace_and_read_only_the_walked_rows(gpu):
+    from paper_2603_08899_b200 import binding as cb
+    cfg = CASES["bf16_noise"]
+    parent, owner = inputs.trees(cfg)
+    tl, dl = inputs.logits(cfg)
+    tok = inputs.draft_tokens(cfg, parent, dl, 1.0)
+    u = inputs.uniforms(cfg)
+    base = H.gpu_accept(gpu, cfg, tl, dl, tok, parent, owner, u, 1.0, 1 | LAZY)
+    bad_t, bad_d = tl.clone(), dl.clone()
+    for b in range(cfg.B):
+        on_path = set(base["path"][b, :base["accept_len"][b].item() + 1].tolist())
+        off = [i for i in range(cfg.T) if i not in on_path]
+        bad_t[b, off[0], 11] = float("nan")
+        bad_d[b, off[-1], cfg.V - 1] = float("inf")
+    dev = "cuda"
+    o = {"accept_len": torch.zeros(cfg.B, dtype=torch.int32, device=dev),
+         "path": torch.zeros((cfg.B, cb.MAX_DEPTH + 1), dtype=torch.int32, device=dev),
+         "next_token": torch.zeros(cfg.B, dtype=torch.int32, device=dev),
+         "status": torch.zeros(cfg.B, dtype=torch.int32, device=dev)}
+    cb.confu_tree_accept(gpu.ctx, cfg.B, cfg.T, cfg.C, cfg.V, tl.dtype, bad_t.to(dev), bad_d.to(dev), tok.to(dev),
+                         parent.to(dev), owner.to(dev), u.to(dev), 1.0, 1 | LAZY, o["accept_len"], o["path"],
+                         o["next_token"], None, None, None, o["status"])          # no workspace
+    torch.cuda.synchronize()
+    assert o["status"].cpu().tolist() == [0] * cfg.B
+    for k in ("accept_len", "path", "next_token"):
+        assert torch.equal(o[k].cpu(), base[k]), k
+    # the default mode sees them
+    got = H.gpu_accept(gpu, cfg, bad_t, bad_d, tok, parent, owner, u, 1.0, 1)
+    assert got["status"].tolist() == [5] * cfg.B
+    # a bad logit on the path is an error in lazy mode too, and agrees with the oracle
+    bad_d = dl.clone()
+    last = base["path"][3, base["accept_len"][3].item()].item()
+    bad_d[3, last, 17] = float("nan")
+    got = H.gpu_accept(gpu, cfg, tl, bad_d, tok, parent, owner, u, 1.0, 1 | LAZY)
+    want = ref.tree_accept(tl, bad_d, tok, parent, owner, u, temperature=1.0, sibling_mode=1 | LAZY)
+    assert got["status"].tolist() == want["status"].tolist() and got["status"][3].item() == 5
+    H.compare_accept(got, want)

@@ -349,3 +349,55 @@ def test_distribution_test_has_power_against_a_dropped_residual_step():
     o = ref.tree_accept(tl, dl, tok, parent, None, u, temperature=1.0, sibling_mode=1)
     first, _ = _emitted(o, tok)
     assert (first == good).all()
+
+
+# ---------------------------------------------------------------- statistics on demand
+LAZY = 0x100
+
+
+def test_lazy_flag_changes_nothing_on_finite_inputs():
+    for seed, temperature, mode in ((41, 1.0, 1), (42, 0.7, 0), (43, 0.0, 1)):
+        cfg, parent, owner, tl, dl, tok, u = _random_case(seed=seed, draft="noise", B=8)
+        if temperature == 0.0:
+            tok = inputs.draft_tokens(cfg, parent, dl, 0.0)
+        a = ref.tree_accept(tl, dl, tok, parent, owner, u, temperature=temperature, sibling_mode=mode)
+        b = ref.tree_accept(tl, dl, tok, parent, owner, u, temperature=temperature, sibling_mode=mode | LAZY)
+        for k in a:
+            assert torch.equal(a[k], b[k]), k
+
+
+def test_lazy_flag_reads_only_the_rows_the_walk_needs():
+    cfg, parent, owner, tl, dl, tok, u = _random_case(seed=44, draft="noise", B=6)
+    base = ref.tree_accept(tl, dl, tok, parent, owner, u, temperature=1.0, sibling_mode=1 | LAZY)
+    assert base["status"].tolist() == [0] * cfg.B
+    for b in range(cfg.B):
+        on_path = set(base["path"][b, :base["accept_len"][b].item() + 1].tolist())
+        off = [i for i in range(cfg.T) if i not in on_path]
+        bad_t, bad_d = tl.clone(), dl.clone()
+        bad_t[b, off[0], 2] = float("nan")
+        bad_d[b, off[-1], 3] = float("inf")
+        o = ref.tree_accept(bad_t, bad_d, tok, parent, owner, u, temperature=1.0, sibling_mode=1 | LAZY)
+        for k in base:
+            assert torch.equal(o[k], base[k]), (b, k)
+        # ... which the default mode reports
+        o = ref.tree_accept(bad_t, bad_d, tok, parent, owner, u, temperature=1.0, sibling_mode=1)
+        assert o["status"][b].item() == ref.ST_NONFINITE
+        # a bad logit in a visited node's draft row is an error in both modes
+        last = base["path"][b, base["accept_len"][b].item()].item()
+        bad_d = dl.clone()
+        bad_d[b, last, 1] = float("-inf")
+        o = ref.tree_accept(tl, bad_d, tok, parent, owner, u, temperature=1.0, sibling_mode=1 | LAZY)
+        assert o["status"][b].item() == ref.ST_NONFINITE and o["next_token"][b].item() == -1
+    # greedy: rows of nodes whose children are never compared are not read
+    tok0 = inputs.draft_tokens(cfg, parent, dl, 0.0)
+    g = ref.tree_accept(tl, None, tok0, parent, owner, None, temperature=0.0, sibling_mode=1 | LAZY)
+    for b in range(cfg.B):
+        kept = set(g["path"][b, :g["accept_len"][b].item() + 1].tolist())
+        dead = [i for i in range(1, cfg.T) if parent[b, i].item() not in kept and i not in kept]
+        leaf_dead = [i for i in dead if not (parent[b] == i).any()]
+        if not leaf_dead:
+            continue
+        bad = tl.clone()
+        bad[b, leaf_dead[0], 0] = float("nan")
+        o = ref.tree_accept(bad, None, tok0, parent, owner, None, temperature=0.0, sibling_mode=1 | LAZY)
+        assert o["status"][b].item() == 0 and torch.equal(o["path"], g["path"])
