@@ -567,3 +567,59 @@ int confu_ref_kv_compact(int32_t B, int32_t n_layers, int64_t row_bytes,
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------ */
+/* contemplate-token embedding: mixture of expert embeddings           */
+/* ------------------------------------------------------------------ */
+int confu_ref_con_embedding(int32_t B, int32_t H_in, int32_t H_out, int32_t n_expert, int32_t k_expert,
+                            int32_t dtype, const void* hidden, const void* router_w, const void* router_b,
+                            const void* experts, int32_t renormalize,
+                            double* out, int32_t* sel, double* gate, double* gap)
+{
+    if (B < 0 || H_in <= 0 || H_out <= 0 || n_expert <= 0 || k_expert <= 0 || k_expert > n_expert) return -1;
+    if (dtype < CONFU_REF_BF16 || dtype > CONFU_REF_F64) return -1;
+    if (!hidden || !router_w || !experts || !out) return -1;
+#pragma omp parallel for schedule(static)
+    for (int b = 0; b < B; ++b) {
+        double* score = (double*)malloc((size_t)n_expert * sizeof(double));
+        int* taken = (int*)calloc((size_t)n_expert, sizeof(int));
+        /* router: a linear layer on the hidden state, then a softmax over the experts */
+        double m = -INFINITY;
+        for (int e = 0; e < n_expert; ++e) {
+            double a = router_b ? load_elem(router_b, dtype, e) : 0.0;
+            for (int i = 0; i < H_in; ++i)
+                a += load_elem(router_w, dtype, (int64_t)e * H_in + i) * load_elem(hidden, dtype, (int64_t)b * H_in + i);
+            score[e] = a;
+            if (a > m) m = a;
+        }
+        double z = 0.0;
+        for (int e = 0; e < n_expert; ++e) { score[e] = exp(score[e] - m); z += score[e]; }
+        for (int e = 0; e < n_expert; ++e) score[e] /= z;
+        /* the k_expert largest scores, largest first, the lower index on equal scores */
+        double wsum = 0.0, kth = 0.0;
+        for (int j = 0; j < H_out; ++j) out[(int64_t)b * H_out + j] = 0.0;
+        int* pick = (int*)malloc((size_t)k_expert * sizeof(int));
+        for (int k = 0; k < k_expert; ++k) {
+            int best = -1;
+            for (int e = 0; e < n_expert; ++e)
+                if (!taken[e] && (best < 0 || score[e] > score[best])) best = e;
+            taken[best] = 1;
+            pick[k] = best;
+            wsum += score[best];
+            kth = score[best];
+        }
+        double next = -INFINITY;
+        for (int e = 0; e < n_expert; ++e) if (!taken[e] && score[e] > next) next = score[e];
+        /* weighted sum of the chosen experts' embeddings, weights = their gating scores */
+        for (int k = 0; k < k_expert; ++k) {
+            const double w = renormalize ? score[pick[k]] / wsum : score[pick[k]];
+            if (sel) sel[(int64_t)b * k_expert + k] = pick[k];
+            if (gate) gate[(int64_t)b * k_expert + k] = w;
+            for (int j = 0; j < H_out; ++j)
+                out[(int64_t)b * H_out + j] += w * load_elem(experts, dtype, (int64_t)pick[k] * H_out + j);
+        }
+        if (gap) gap[b] = k_expert < n_expert ? kth - next : INFINITY;
+        free(score); free(taken); free(pick);
+    }
+    return 0;
+}

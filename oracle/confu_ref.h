@@ -160,6 +160,24 @@ int confu_ref_kv_compact(int32_t B, int32_t n_layers, int64_t row_bytes,
                          const int32_t* accept_len, const int32_t* path,
                          int32_t* new_prefix_len);
 
+/*
+ * Embedding of the contemplate token as a mixture of expert embeddings (Sec. 3.2,
+ * "Dynamic Contemplate Tokens with MoE"): a linear layer maps the hidden state of
+ * the most recently accepted token to one logit per expert (router_w
+ * [n_expert][H_in], optional bias router_b [n_expert]), a softmax normalises them,
+ * the k_expert experts with the largest scores are selected (the lower index on
+ * equal scores) and the embedding is the sum of their embeddings (experts
+ * [n_expert][H_out]) weighted by their gating scores -- the softmax values
+ * themselves, or, with renormalize != 0, divided by their sum over the selection.
+ * hidden [B][H_in]; out [B][H_out] doubles; optional: sel [B][k_expert] (largest
+ * score first), gate [B][k_expert] (the weights used), gap [B] = score of the last
+ * selected expert minus the largest score left out (+inf if none is left out).
+ */
+int confu_ref_con_embedding(int32_t B, int32_t H_in, int32_t H_out, int32_t n_expert, int32_t k_expert,
+                            int32_t dtype, const void* hidden, const void* router_w, const void* router_b,
+                            const void* experts, int32_t renormalize,
+                            double* out, int32_t* sel, double* gate, double* gap);
+
 /* number of OpenMP threads the oracle will use */
 int confu_ref_num_threads(void);
 

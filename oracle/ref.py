@@ -37,7 +37,8 @@ def lib():
         _lib = C.CDLL(_build.build())
         _lib.confu_ref_num_threads.restype = C.c_int
         for name in ("confu_ref_tree_attention", "confu_ref_tree_attention_rows",
-                     "confu_ref_tree_accept", "confu_ref_tree_accept_match", "confu_ref_kv_compact"):
+                     "confu_ref_tree_accept", "confu_ref_tree_accept_match", "confu_ref_kv_compact",
+                     "confu_ref_con_embedding"):
             getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -192,3 +193,24 @@ def kv_compact(k_layers, v_layers, seq_start, prefix_len, accept_len, path):
     if rc != 0:
         raise ValueError("confu_ref_kv_compact: bad argument")
     return new_len
+
+
+def con_embedding(hidden, router_w, router_b, experts, k_expert, renormalize=False):
+    """Mixture-of-experts embedding of the contemplate token.  Returns (out [B,H_out] fp64,
+    sel [B,k] int32, gate [B,k] fp64, gap [B] fp64)."""
+    B, H_in = hidden.shape
+    n_expert, H_out = experts.shape
+    dt = hidden.dtype
+    assert router_w.dtype == dt and experts.dtype == dt and (router_b is None or router_b.dtype == dt)
+    out = torch.zeros(B, H_out, dtype=torch.float64)
+    sel = torch.zeros(B, k_expert, dtype=torch.int32)
+    gate = torch.zeros(B, k_expert, dtype=torch.float64)
+    gap = torch.zeros(B, dtype=torch.float64)
+    rb = None if router_b is None else router_b.contiguous()
+    rc = lib().confu_ref_con_embedding(C.c_int32(B), C.c_int32(H_in), C.c_int32(H_out), C.c_int32(n_expert),
+                                       C.c_int32(k_expert), C.c_int32(_DT[dt]), _p(hidden.contiguous()),
+                                       _p(router_w.contiguous()), _p(rb), _p(experts.contiguous()),
+                                       C.c_int32(1 if renormalize else 0), _p(out), _p(sel), _p(gate), _p(gap))
+    if rc != 0:
+        raise ValueError("confu_ref_con_embedding: bad argument")
+    return out, sel, gate, gap
