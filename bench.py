@@ -326,6 +326,35 @@ def run_ours(args, cfg):
     ms_plan, ms_attn, ms_acc, ms_cmp = part(0, 1), part(1, 2), part(2, 3), part(3, 4)
     alen = step.accept_len.float().mean().item()
 
+    def time_accept_variants():
+        """Outside the timed step: the acceptance variants that read only the walked path's rows.
+        ms per call, and the logit bytes each one actually reads (from its own accepted lengths)."""
+        out = {}
+        for name in ("lazy", "match"):
+            def call():
+                if name == "lazy":
+                    step.run_accept(1.0, 1 | cb.ACCEPT_LAZY)
+                else:
+                    cb.confu_tree_accept_match(step.ctx, cfg.B, cfg.T, cfg.C, cfg.V, cfg.logit_dtype, step.tl, step.tokens,
+                                               step.parent, step.con_owner, step.uniforms, 1.0, step.accept_len, step.path,
+                                               step.next_token, step.future_row, step.counters, step.status)
+            call()
+            torch.cuda.synchronize()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+            for i in range(5):
+                e[i].record()
+                call()
+            e[5].record()
+            torch.cuda.synchronize()
+            rows = (step.accept_len.long() + 1).sum().item() * (2 if name == "lazy" else 1)
+            out[name] = {"ms": e[0].elapsed_time(e[5]) / 5, "logit_bytes_read": rows * cfg.V * step.tl.element_size(),
+                         "mean_accept_len": step.accept_len.float().mean().item()}
+        step.run_accept(1.0)                      # leave the default rule's results in place
+        torch.cuda.synchronize()
+        return out
+
+    accept_variants = time_accept_variants() if rank == 0 else None
+
     def measure_e2e():
         # ---- end to end: this step's inputs come from pinned host memory, results go back ----
         h = {"q": [t.cpu().pin_memory() for t in step.q],
@@ -424,6 +453,9 @@ def run_ours(args, cfg):
                    "l2": "inputs larger than L2 (every layer has its own KV; no flush needed)",
                    "parallelism": f"replicas x{world}, sequences sharded, no collective",
                    "parts_ms": {"plan": ms_plan, "attention": ms_attn, "accept": ms_acc, "compact": ms_cmp},
+                   "accept_rule": "ratio test, statistics of all rows (timed); variants timed apart: " \
+                                  "lazy = same rule, rows on demand; match = sample-and-match, rows on demand",
+                   "accept_variants": accept_variants,
                    "step_bytes": sbytes, "step_gbs": sbytes / (ms_step * 1e-3) / 1e9,
                    "step_frac_of_hbm_roofline": sbytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                    "mean_accept_len": alen, "status_ok": status_ok, "spot_check_vs_oracle": checked},

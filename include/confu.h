@@ -270,6 +270,27 @@ int confu_kv_append(confu_ctx* ctx, const confu_dims* dims, const void* k_rows, 
                     void* k_cache, void* v_cache, const int64_t* seq_start, const int32_t* prefix_len,
                     void* stream);
 
+/* ---- contemplate-token embedding (Sec. 3.2, "Dynamic Contemplate Tokens with MoE") ---- */
+
+/*
+ * The embedding of the contemplate token that the verification forward feeds to the target model,
+ * as a mixture of n_expert learnable embeddings conditioned on the hidden state of the most
+ * recently accepted token: a linear layer (router_w [n_expert][H_in], optional bias router_b
+ * [n_expert]) maps hidden [B][H_in] to one logit per expert, a softmax normalises them, the
+ * k_expert largest scores are selected (the lower index on equal scores) and
+ *   out[b][:] = sum over the selection of  gate * experts[e][:]        (experts [n_expert][H_out])
+ * with gate = the expert's softmax score, or, with renormalize != 0, that score divided by the sum
+ * over the selection (the paper says "normalized gating scores" and does not say which; it gives
+ * neither n_expert nor k_expert: both are arguments; limits n_expert <= 1024, k_expert <= 32).
+ * All five tensors have the type `dtype` (CONFU_BF16 | CONFU_F32), rows contiguous; accumulation
+ * is fp32.  Optional outputs: sel [B][k_expert] int32 (largest score first) and gate [B][k_expert]
+ * fp32 (the weights used).  All pointers device, 16-byte aligned.
+ */
+int confu_con_embedding(confu_ctx* ctx, int32_t B, int32_t H_in, int32_t H_out, int32_t n_expert, int32_t k_expert,
+                        int32_t dtype, const void* hidden, const void* router_w, const void* router_b,
+                        const void* experts, int32_t renormalize, void* out, int32_t* sel, float* gate,
+                        void* stream);
+
 #ifdef __cplusplus
 }
 #endif

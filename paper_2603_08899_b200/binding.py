@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(HERE, "libconfu.so")
 MAX_TREE = 64
 MAX_ROWS = 128
 MAX_DEPTH = 63
+ACCEPT_LAZY = 0x100          # or-ed into sibling_mode: row statistics on demand
 BF16, F32 = 0, 1
 OK = 0
 
@@ -23,7 +24,7 @@ EXPORTS = [
     "confu_last_cuda_error", "confu_plan_bytes", "confu_tree_plan", "confu_tree_attention",
     "confu_accept_workspace_bytes", "confu_tree_accept", "confu_kv_compact", "confu_kv_append",
     "confu_tree_accept_static_max_rows", "confu_tree_accept_static", "confu_set_paging",
-    "confu_tree_accept_match",
+    "confu_tree_accept_match", "confu_con_embedding",
 ]
 
 
@@ -51,7 +52,7 @@ def lib():
         L.confu_last_cuda_error.restype = C.c_char_p
         for n in ("confu_create", "confu_destroy", "confu_set_workspace", "confu_tree_plan", "confu_tree_attention",
                   "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static", "confu_set_paging",
-                  "confu_tree_accept_match"):
+                  "confu_tree_accept_match", "confu_con_embedding"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -162,6 +163,18 @@ def confu_tree_accept_match(ctx, B, T, Cn, V, logit_dtype, target_logits, tokens
                                          _ptr(parent), _ptr(con_owner), _ptr(uniforms), C.c_float(temperature),
                                          _ptr(accept_len), _ptr(path), _ptr(next_token), _ptr(future_row),
                                          _ptr(counters), _ptr(status), _stream(stream)), ctx)
+
+
+def confu_con_embedding(ctx, hidden, router_w, router_b, experts, k_expert, renormalize, out, sel=None, gate=None,
+                        stream=None):
+    """Contemplate-token embedding: router -> softmax -> top-k experts -> weighted sum of their embeddings."""
+    B, H_in = hidden.shape
+    n_expert, H_out = experts.shape
+    _check("confu_con_embedding",
+           lib().confu_con_embedding(ctx, C.c_int32(B), C.c_int32(H_in), C.c_int32(H_out), C.c_int32(n_expert),
+                                     C.c_int32(k_expert), C.c_int32(dtype_code(hidden.dtype)), _ptr(hidden),
+                                     _ptr(router_w), _ptr(router_b), _ptr(experts), C.c_int32(1 if renormalize else 0),
+                                     _ptr(out), _ptr(sel), _ptr(gate), _stream(stream)), ctx)
 
 
 def confu_tree_accept_static_max_rows():

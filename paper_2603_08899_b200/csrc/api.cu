@@ -277,4 +277,20 @@ int confu_kv_append(confu_ctx* ctx, const confu_dims* dims, const void* k_rows, 
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
 }
 
+int confu_con_embedding(confu_ctx* ctx, int32_t B, int32_t H_in, int32_t H_out, int32_t n_expert, int32_t k_expert,
+                        int32_t dtype, const void* hidden, const void* router_w, const void* router_b,
+                        const void* experts, int32_t renormalize, void* out, int32_t* sel, float* gate, void* stream)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    if (B < 0 || H_in <= 0 || H_out <= 0 || n_expert <= 0 || k_expert <= 0 || k_expert > n_expert) return CONFU_ERR_SHAPE;
+    if (dtype != CONFU_BF16 && dtype != CONFU_F32) return CONFU_ERR_ARG;
+    if (n_expert > 1024 || k_expert > 32) return CONFU_ERR_UNSUPPORTED;
+    if (B == 0) return CONFU_OK;
+    if (!hidden || !router_w || !experts || !out) return CONFU_ERR_ARG;
+    if (misaligned(hidden) || misaligned(router_w) || misaligned(experts) || misaligned(out)) return CONFU_ERR_ALIGN;
+    cudaError_t e = launch_con_embedding(B, H_in, H_out, n_expert, k_expert, dtype, hidden, router_w, router_b, experts,
+                                         renormalize != 0, out, sel, gate, (cudaStream_t)stream);
+    return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
+}
+
 }  // extern "C"

@@ -3,6 +3,7 @@
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <limits.h>
 #include <stdint.h>
 
 #include "confu.h"
@@ -189,6 +190,10 @@ cudaError_t launch_compact(const Ctx* ctx, int B, int n_layers, int64_t row_byte
                            void* const* v_layers, const SlotMap& map, const int32_t* prefix_len,
                            const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len,
                            int32_t* status, cudaStream_t st);
+
+cudaError_t launch_con_embedding(int B, int H_in, int H_out, int n_expert, int k_expert, int dtype, const void* hidden,
+                                 const void* router_w, const void* router_b, const void* experts, int renormalize,
+                                 void* out, int32_t* sel, float* gate, cudaStream_t st);
 
 cudaError_t launch_append(int B, int R, int64_t row_bytes, const void* k_rows, const void* v_rows, void* k_cache,
                           void* v_cache, const SlotMap& map, const int32_t* prefix_len, cudaStream_t st);
