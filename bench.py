@@ -296,6 +296,14 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
     checked = spot_check(cfg, step, host) if rank == 0 else True
     status_ok = bool((step.status == 0).all().item())
+    # The timed steps replay the step's launches from CUDA graphs captured here (the same kernels with
+    # the same arguments; the host then issues 4 graph launches per step instead of 2 L + 4 kernels).
+    use_graph = not args.no_graph
+    if use_graph:
+        step.capture(1.0)
+        for _ in range(2):
+            step.replay()
+        torch.cuda.synchronize()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     sampler = ClockSampler(local) if rank == 0 else None
     barrier()
@@ -303,15 +311,13 @@ def run_ours(args, cfg):
     t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record()
     for i in range(args.steps):
+        if use_graph:
+            step.replay(ev[i])
+            continue
         ev[i][0].record()
-        cb.confu_tree_plan(step.ctx, step.dims, step.seq_start, step.prefix_len, step.parent, step.con_owner,
-                           step.plan, step.status)
+        step.run_plan()
         ev[i][1].record()
-        for l in range(cfg.L):
-            cb.confu_tree_attention(step.ctx, step.dims, step.q[l], step.k[l], step.v[l], step.n_slots,
-                                    step.seq_start, step.prefix_len, step.ks[l] if step.ks else None,
-                                    step.vs[l] if step.vs else None, None, None, step.plan, step.out[l], None,
-                                    step.status)
+        step.run_layers()
         ev[i][2].record()
         step.run_accept(1.0)
         ev[i][3].record()
@@ -453,6 +459,8 @@ def run_ours(args, cfg):
                    "l2": "inputs larger than L2 (every layer has its own KV; no flush needed)",
                    "parallelism": f"replicas x{world}, sequences sharded, no collective",
                    "parts_ms": {"plan": ms_plan, "attention": ms_attn, "accept": ms_acc, "compact": ms_cmp},
+                   "launch": "4 CUDA graphs per step (plan | L attention layers | acceptance | compaction)" if use_graph
+                             else "kernel launches from the host, one by one",
                    "accept_rule": "ratio test, statistics of all rows (timed); variants timed apart: " \
                                   "lazy = same rule, rows on demand; match = sample-and-match, rows on demand",
                    "accept_variants": accept_variants,
@@ -489,6 +497,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="batch32", choices=list(inputs.CONFIGS))
+    ap.add_argument("--no-graph", action="store_true", help="time kernel launches issued one by one from the host")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer count (profiling runs; named in config.workload)")

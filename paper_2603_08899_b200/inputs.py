@@ -71,6 +71,11 @@ CONFIGS = {
                                prefix=4096, tree="random", kv_dtype=torch.bfloat16,
                                logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",
                                temperatures=(1.0,), seed=6),
+    # the size Sec. 3.1 calls typical: a draft tree of 30 nodes, one contemplate row each
+    "llama8b_30": VerifyConfig("llama8b_30", B=1, L=32, Hq=32, Hkv=8, D=128, T=30, C=30, S=16, V=128256,
+                               prefix=4096, tree="random", kv_dtype=torch.bfloat16,
+                               logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",
+                               temperatures=(1.0,), seed=8),
     "batch32_2t": VerifyConfig("batch32_2t", B=32, L=32, Hq=32, Hkv=8, D=128, T=60, C=60, S=16, V=128256,
                                prefix=(512, 16384), tree="random", kv_dtype=torch.bfloat16,
                                logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",

@@ -55,6 +55,42 @@ class VerifyStep:
                                     None, None, self.plan, self.out[l],
                                     None if lse_layers is None else lse_layers[l], self.status)
 
+    def run_plan(self):
+        cb.confu_tree_plan(self.ctx, self.dims, self.seq_start, self.prefix_len, self.parent, self.con_owner,
+                           self.plan, self.status)
+
+    def run_layers(self):
+        """The L attention calls with the plan built by run_plan()."""
+        for l in range(len(self.q)):
+            cb.confu_tree_attention(self.ctx, self.dims, self.q[l], self.k[l], self.v[l], self.n_slots,
+                                    self.seq_start, self.prefix_len,
+                                    self.ks[l] if self.ks is not None else None,
+                                    self.vs[l] if self.vs is not None else None,
+                                    None, None, self.plan, self.out[l], None, self.status)
+
+    def capture(self, temperature=1.0, sibling_mode=1):
+        """Record the step's launches once as four CUDA graphs (plan | attention layers | acceptance |
+        compaction) over the bound tensors; replay() then enqueues a step with four graph launches
+        instead of 2 L + 4 kernel launches from the host.  Run the step once before capturing (the
+        first call of each kernel sets function attributes, which a capture does not allow)."""
+        parts = (self.run_plan, self.run_layers, lambda: self.run_accept(temperature, sibling_mode), self.run_compact)
+        self.graphs = []
+        for fn in parts:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            self.graphs.append(g)
+
+    def replay(self, events=None):
+        """Enqueue one captured step on the current stream; events: optional 5 CUDA events recorded
+        before the first graph and after each of the four."""
+        if events is not None:
+            events[0].record()
+        for i, g in enumerate(self.graphs):
+            g.replay()
+            if events is not None:
+                events[i + 1].record()
+
     def run_accept(self, temperature, sibling_mode=1):
         cfg = self.cfg
         cb.confu_tree_accept(self.ctx, cfg.B, cfg.T, cfg.C, cfg.V, cfg.logit_dtype, self.tl,

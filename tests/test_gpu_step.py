@@ -195,3 +195,51 @@ def test_two_chained_steps_through_compaction_and_append():
                                       parent2, owner2)
         H.assert_attention_close(out2.cpu(), lse2.cpu(), w, wl, cfg.kv_dtype, f"second step layer {l}")
     step.close()
+
+
+def test_captured_step_replays_to_the_same_results():
+    """The step captured as CUDA graphs (what the benchmark times) writes the same bits as the
+    launches issued one by one, also after the inputs behind the bound pointers have changed."""
+    cfg = inputs.scaled(inputs.CONFIGS["llama8b"], B=3, L=2, prefix=(100, 700), V=4096)
+    parent, owner, plen, seq_start, n_slots, lt, tl, dl, tok, u = _build(cfg, 2, 1.0)
+    step = VerifyStep(cfg, n_slots)
+    outs = [torch.empty_like(t["q"]) for t in lt]
+    step.bind([t["q"] for t in lt], [t["k_cache"] for t in lt], [t["v_cache"] for t in lt],
+              [t["k_soft"] for t in lt], [t["v_soft"] for t in lt], outs, seq_start.cuda(), plen.cuda(), parent.cuda(),
+              owner.cuda(), tl, dl, tok.cuda(), u.cuda())
+    keep = [(t["k_cache"].clone(), t["v_cache"].clone()) for t in lt]
+
+    def restore():
+        for t, (k, v) in zip(lt, keep):
+            t["k_cache"].copy_(k)
+            t["v_cache"].copy_(v)
+
+    def snapshot():
+        torch.cuda.synchronize()
+        return [o.clone() for o in outs] + [step.accept_len.clone(), step.path.clone(), step.next_token.clone(),
+                                            step.future_row.clone(), step.new_prefix_len.clone(), step.status.clone()] + \
+               [t["k_cache"].clone() for t in lt]
+
+    step.run(1.0)
+    eager = snapshot()
+    restore()
+    step.capture(1.0)
+    restore()                                   # (a capture does not run the kernels; this is for symmetry)
+    for o in outs:
+        o.zero_()
+    step.accept_len.fill_(-1)
+    step.replay()
+    for a, b in zip(eager, snapshot()):
+        assert torch.equal(a, b)
+    # new queries behind the same pointers: replay follows, eager agrees
+    restore()
+    for t in lt:
+        t["q"].copy_(torch.roll(t["q"], 1, dims=1))
+    step.replay()
+    replayed = snapshot()
+    restore()
+    step.run(1.0)
+    for a, b in zip(snapshot(), replayed):
+        assert torch.equal(a, b)
+    assert not torch.equal(replayed[0], eager[0])
+    step.close()
