@@ -62,13 +62,15 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
 
 
-KERNEL_SOURCES = {"attention_tc_kernel": "attn_tc.cu", "attention_generic_kernel": "attn_generic.cu"}
+KERNEL_SOURCES = {"attention_tc_kernel": ("attn_tc.cu", "attn_tc.cuh"), "attention_generic_kernel": ("attn_generic.cu",)}
 
 
 def kernel_source_hash(kernel):
     import hashlib
-    src = os.path.join(ROOT, "paper_2603_08899_b200", "csrc", KERNEL_SOURCES[kernel])
-    return hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kernel]:
+        h.update(open(os.path.join(ROOT, "paper_2603_08899_b200", "csrc", name), "rb").read())
+    return h.hexdigest()[:16]
 
 
 def profile_traffic(kernel, workload):

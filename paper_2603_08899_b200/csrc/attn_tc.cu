@@ -23,7 +23,7 @@
 #include <cuda.h>
 #include <stdlib.h>
 
-#include "common.cuh"
+#include "attn_tc.cuh"
 
 namespace confu {
 
@@ -31,7 +31,6 @@ namespace tc {
 
 constexpr int kThreads = 384;            // warps 0-3: softmax of M tile 0, 4-7: of M tile 1, 8: TMA, 9: MMA
 constexpr int kStages = 2;               // ring of stages; stage g = [V of the CTA's g-1st key tile | K of its g-th]
-constexpr int kD = 128;
 constexpr int kTileBytes = kTileKeys * kD * 2;      // 32 KB
 constexpr int kHalfTile = kTileBytes / 2;           // one 64-wide half of the head dim: [128 rows][128 B]
 constexpr int kQBytes = 2 * kTileBytes;             // two M tiles
@@ -47,21 +46,6 @@ struct SharedStorage {
     uint64_t s_full[2], p_full[2], o_done[2];
     uint32_t tmem_base;
     int abort;
-};
-
-struct Params {
-    confu_dims d;
-    SlotMap map;         // packed pool (seq_start) or paged pool (block table, pages of 128 slots = one key tile)
-    const int32_t* prefix_len;
-    const void* plan;
-    float* partials;
-    __nv_bfloat16* out;
-    float* lse;
-    int32_t* status;
-    int n_mt;            // M tiles in use (R > 32 ? 2 : 1)
-    int n_rg;            // groups of 64 query rows (R > 64 ? 2 : 1); a pair = (sequence, kv head, row group)
-    int G;
-    float c;             // sm_scale * log2(e)
 };
 
 // ------------------------------------------------------------------------------------ PTX wrappers
@@ -179,13 +163,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
           "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
           "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
         : "memory");
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
 }
 
 // Low word of a shared-memory matrix descriptor: start address and leading byte offset, both >> 4.
@@ -647,129 +624,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     }
 }
 
-// Merge of the split-KV partials of one (sequence, kv head) pair, in CTA order (deterministic).
-// One block per (pair, M tile, 32 rows); a warp takes a row at a time (four rows in all), lane i the
-// row's columns 4i..4i+3, so partial rows are read and output rows written as whole 512- and
-// 256-byte lines.
-__global__ void __launch_bounds__(256) combine_kernel(const Params prm)
-{
-    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
-    const int pair = blockIdx.x, t = blockIdx.y;
-    // pairs: sequence major, then kv head, then row group
-    const int per_seq = prm.d.Hkv * prm.n_rg;
-    const int b = pair / per_seq, g = (pair % per_seq) / prm.n_rg, rg = pair % prm.n_rg;
-    const int nt = pv.tiles[b];
-    if (nt == 0 || t >= prm.n_mt) return;
-    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
-    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
-    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
-    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
-    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
-    const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const size_t slot_floats = partial_slot_bytes() / sizeof(float);
-    for (int lane_row = blockIdx.z * 32 + warp; lane_row < min(32 * G, (int)blockIdx.z * 32 + 32); lane_row += 8) {
-        const int r = kGroupRows * rg + 32 * t + lane_row / G, hl = lane_row % G;
-        if (r >= R) break;
-        const int row = t * 128 + lane_row;
-        float M = -INFINITY;
-        for (int cta = c_first; cta <= c_last; ++cta) {
-            const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
-            M = fmaxf(M, slot[(size_t)kPartRows * kPartD + row]);
-        }
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float L = 0.f;
-        for (int cta = c_first; cta <= c_last; ++cta) {
-            const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
-            const float m = slot[(size_t)kPartRows * kPartD + row];
-            const float w = (m == -INFINITY) ? 0.f : ex2(m - M);
-            L += w * slot[(size_t)kPartRows * kPartD + kPartRows + row];
-            const float4 v = reinterpret_cast<const float4*>(slot + (size_t)row * kPartD)[lane];
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
-        }
-        const float inv_l = 1.f / L;
-        const int h = g * G + hl;
-        __nv_bfloat16* orow = prm.out + (((size_t)b * R + r) * Hq + h) * kD;
-        uint2 pkt;
-        pkt.x = pack_bf16(acc.x * inv_l, acc.y * inv_l);
-        pkt.y = pack_bf16(acc.z * inv_l, acc.w * inv_l);
-        reinterpret_cast<uint2*>(orow)[lane] = pkt;
-        if (prm.lse && lane == 0) prm.lse[((size_t)b * R + r) * Hq + h] = (M + log2f(L)) * 0.6931471805599453f;
-    }
-}
-
-// The same merge for pairs spread over many CTAs (long prefixes in a small batch: more CTAs than
-// pairs).  One block per (pair, M tile, 16 rows), one warp per row; the parts' maxima and weights are
-// taken 32 parts at a time, one per lane, and the rows of eight parts are in flight together.  The
-// order of every sum is fixed by the part index alone, so the result does not depend on the run.
-constexpr int kCombineRowsPerBlock = 16;
-__global__ void __launch_bounds__(32 * kCombineRowsPerBlock) combine_wide_kernel(const Params prm)
-{
-    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
-    const int pair = blockIdx.x, t = blockIdx.y;
-    // pairs: sequence major, then kv head, then row group
-    const int per_seq = prm.d.Hkv * prm.n_rg;
-    const int b = pair / per_seq, g = (pair % per_seq) / prm.n_rg, rg = pair % prm.n_rg;
-    const int nt = pv.tiles[b];
-    if (nt == 0 || t >= prm.n_mt) return;
-    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
-    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
-    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
-    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
-    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
-    const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int lane_row = blockIdx.z * kCombineRowsPerBlock + warp;
-    const int r = kGroupRows * rg + 32 * t + lane_row / G, hl = lane_row % G;
-    if (lane_row >= 32 * G || r >= R) return;
-    const int row = t * 128 + lane_row;
-    const int n_parts = c_last - c_first + 1;
-    const size_t slot_floats = partial_slot_bytes() / sizeof(float);
-    auto slot_of = [&](int p) {                         // part p of the pair: the partial slot of CTA c_first + p
-        const int cta = c_first + p;
-        return prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
-    };
-    float M = -INFINITY;
-    for (int p = lane; p < n_parts; p += 32) M = fmaxf(M, slot_of(p)[(size_t)kPartRows * kPartD + row]);
-    M = warp_max(M);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float L = 0.f;
-    for (int p0 = 0; p0 < n_parts; p0 += 32) {
-        float w = 0.f, wl = 0.f;                        // this lane's part of the group: weight, weight * sum
-        if (p0 + lane < n_parts) {
-            const float* ml = slot_of(p0 + lane) + (size_t)kPartRows * kPartD;
-            const float m = ml[row];
-            w = (m == -INFINITY) ? 0.f : ex2(m - M);
-            wl = w * ml[kPartRows + row];
-        }
-        L += warp_sum(wl);
-        const int n_grp = min(32, n_parts - p0);
-        for (int q0 = 0; q0 < n_grp; q0 += 8) {
-            float4 v[8];
-            float wq[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                wq[k] = __shfl_sync(0xffffffffu, w, (q0 + k) & 31);      // 0 past the last part
-                v[k] = q0 + k < n_grp ? reinterpret_cast<const float4*>(slot_of(p0 + q0 + k) + (size_t)row * kPartD)[lane]
-                                      : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                acc.x = fmaf(wq[k], v[k].x, acc.x); acc.y = fmaf(wq[k], v[k].y, acc.y);
-                acc.z = fmaf(wq[k], v[k].z, acc.z); acc.w = fmaf(wq[k], v[k].w, acc.w);
-            }
-        }
-    }
-    const float inv_l = 1.f / L;
-    const int h = g * G + hl;
-    __nv_bfloat16* orow = prm.out + (((size_t)b * R + r) * Hq + h) * kD;
-    uint2 pkt;
-    pkt.x = pack_bf16(acc.x * inv_l, acc.y * inv_l);
-    pkt.y = pack_bf16(acc.z * inv_l, acc.w * inv_l);
-    reinterpret_cast<uint2*>(orow)[lane] = pkt;
-    if (prm.lse && lane == 0) prm.lse[((size_t)b * R + r) * Hq + h] = (M + log2f(L)) * 0.6931471805599453f;
-}
-
 // ------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -849,13 +703,7 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     attention_tc_kernel<<<ctx->sm_count, kThreads, smem, st>>>(q_map, k_map, v_map, ks_map, vs_map, prm);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    // few pairs for the machine (each spread over several CTAs): the merge that is parallel over parts
-    const int n_pairs = d.B * d.Hkv * prm.n_rg;
-    if (ctx->sm_count >= 2 * n_pairs)
-        combine_wide_kernel<<<dim3(n_pairs, prm.n_mt, 128 / kCombineRowsPerBlock), 32 * kCombineRowsPerBlock, 0, st>>>(prm);
-    else
-        combine_kernel<<<dim3(n_pairs, prm.n_mt, 4), 256, 0, st>>>(prm);
-    return cudaGetLastError();
+    return launch_combine(prm, ctx->sm_count, st);
 }
 
 }  // namespace confu

@@ -1,0 +1,144 @@
+// Merge of the split-KV partial results of the tensor-core attention kernel: a pair (sequence, kv
+// head, row group) whose key tiles were walked by several CTAs has one unnormalised partial (O, m,
+// l) per CTA; these kernels combine them into the output rows.
+#include "attn_tc.cuh"
+
+namespace confu {
+namespace tc {
+
+// Merge of the split-KV partials of one (sequence, kv head) pair, in CTA order (deterministic).
+// One block per (pair, M tile, 32 rows); a warp takes a row at a time (four rows in all), lane i the
+// row's columns 4i..4i+3, so partial rows are read and output rows written as whole 512- and
+// 256-byte lines.
+__global__ void __launch_bounds__(256) combine_kernel(const Params prm)
+{
+    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
+    const int pair = blockIdx.x, t = blockIdx.y;
+    // pairs: sequence major, then kv head, then row group
+    const int per_seq = prm.d.Hkv * prm.n_rg;
+    const int b = pair / per_seq, g = (pair % per_seq) / prm.n_rg, rg = pair % prm.n_rg;
+    const int nt = pv.tiles[b];
+    if (nt == 0 || t >= prm.n_mt) return;
+    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
+    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
+    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
+    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
+    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
+    const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t slot_floats = partial_slot_bytes() / sizeof(float);
+    for (int lane_row = blockIdx.z * 32 + warp; lane_row < min(32 * G, (int)blockIdx.z * 32 + 32); lane_row += 8) {
+        const int r = kGroupRows * rg + 32 * t + lane_row / G, hl = lane_row % G;
+        if (r >= R) break;
+        const int row = t * 128 + lane_row;
+        float M = -INFINITY;
+        for (int cta = c_first; cta <= c_last; ++cta) {
+            const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
+            M = fmaxf(M, slot[(size_t)kPartRows * kPartD + row]);
+        }
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float L = 0.f;
+        for (int cta = c_first; cta <= c_last; ++cta) {
+            const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
+            const float m = slot[(size_t)kPartRows * kPartD + row];
+            const float w = (m == -INFINITY) ? 0.f : ex2(m - M);
+            L += w * slot[(size_t)kPartRows * kPartD + kPartRows + row];
+            const float4 v = reinterpret_cast<const float4*>(slot + (size_t)row * kPartD)[lane];
+            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+        }
+        const float inv_l = 1.f / L;
+        const int h = g * G + hl;
+        __nv_bfloat16* orow = prm.out + (((size_t)b * R + r) * Hq + h) * kD;
+        uint2 pkt;
+        pkt.x = pack_bf16(acc.x * inv_l, acc.y * inv_l);
+        pkt.y = pack_bf16(acc.z * inv_l, acc.w * inv_l);
+        reinterpret_cast<uint2*>(orow)[lane] = pkt;
+        if (prm.lse && lane == 0) prm.lse[((size_t)b * R + r) * Hq + h] = (M + log2f(L)) * 0.6931471805599453f;
+    }
+}
+
+// The same merge for pairs spread over many CTAs (long prefixes in a small batch: more CTAs than
+// pairs).  One block per (pair, M tile, 16 rows), one warp per row; the parts' maxima and weights are
+// taken 32 parts at a time, one per lane, and the rows of eight parts are in flight together.  The
+// order of every sum is fixed by the part index alone, so the result does not depend on the run.
+constexpr int kCombineRowsPerBlock = 16;
+__global__ void __launch_bounds__(32 * kCombineRowsPerBlock) combine_wide_kernel(const Params prm)
+{
+    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
+    const int pair = blockIdx.x, t = blockIdx.y;
+    // pairs: sequence major, then kv head, then row group
+    const int per_seq = prm.d.Hkv * prm.n_rg;
+    const int b = pair / per_seq, g = (pair % per_seq) / prm.n_rg, rg = pair % prm.n_rg;
+    const int nt = pv.tiles[b];
+    if (nt == 0 || t >= prm.n_mt) return;
+    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
+    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
+    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
+    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
+    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
+    const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lane_row = blockIdx.z * kCombineRowsPerBlock + warp;
+    const int r = kGroupRows * rg + 32 * t + lane_row / G, hl = lane_row % G;
+    if (lane_row >= 32 * G || r >= R) return;
+    const int row = t * 128 + lane_row;
+    const int n_parts = c_last - c_first + 1;
+    const size_t slot_floats = partial_slot_bytes() / sizeof(float);
+    auto slot_of = [&](int p) {                         // part p of the pair: the partial slot of CTA c_first + p
+        const int cta = c_first + p;
+        return prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
+    };
+    float M = -INFINITY;
+    for (int p = lane; p < n_parts; p += 32) M = fmaxf(M, slot_of(p)[(size_t)kPartRows * kPartD + row]);
+    M = warp_max(M);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    for (int p0 = 0; p0 < n_parts; p0 += 32) {
+        float w = 0.f, wl = 0.f;                        // this lane's part of the group: weight, weight * sum
+        if (p0 + lane < n_parts) {
+            const float* ml = slot_of(p0 + lane) + (size_t)kPartRows * kPartD;
+            const float m = ml[row];
+            w = (m == -INFINITY) ? 0.f : ex2(m - M);
+            wl = w * ml[kPartRows + row];
+        }
+        L += warp_sum(wl);
+        const int n_grp = min(32, n_parts - p0);
+        for (int q0 = 0; q0 < n_grp; q0 += 8) {
+            float4 v[8];
+            float wq[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                wq[k] = __shfl_sync(0xffffffffu, w, (q0 + k) & 31);      // 0 past the last part
+                v[k] = q0 + k < n_grp ? reinterpret_cast<const float4*>(slot_of(p0 + q0 + k) + (size_t)row * kPartD)[lane]
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                acc.x = fmaf(wq[k], v[k].x, acc.x); acc.y = fmaf(wq[k], v[k].y, acc.y);
+                acc.z = fmaf(wq[k], v[k].z, acc.z); acc.w = fmaf(wq[k], v[k].w, acc.w);
+            }
+        }
+    }
+    const float inv_l = 1.f / L;
+    const int h = g * G + hl;
+    __nv_bfloat16* orow = prm.out + (((size_t)b * R + r) * Hq + h) * kD;
+    uint2 pkt;
+    pkt.x = pack_bf16(acc.x * inv_l, acc.y * inv_l);
+    pkt.y = pack_bf16(acc.z * inv_l, acc.w * inv_l);
+    reinterpret_cast<uint2*>(orow)[lane] = pkt;
+    if (prm.lse && lane == 0) prm.lse[((size_t)b * R + r) * Hq + h] = (M + log2f(L)) * 0.6931471805599453f;
+}
+
+cudaError_t launch_combine(const Params& prm, int sm_count, cudaStream_t st)
+{
+    // few pairs for the machine (each spread over several CTAs): the merge that is parallel over parts
+    const int n_pairs = prm.d.B * prm.d.Hkv * prm.n_rg;
+    if (sm_count >= 2 * n_pairs)
+        combine_wide_kernel<<<dim3(n_pairs, prm.n_mt, 128 / kCombineRowsPerBlock), 32 * kCombineRowsPerBlock, 0, st>>>(prm);
+    else
+        combine_kernel<<<dim3(n_pairs, prm.n_mt, 4), 256, 0, st>>>(prm);
+    return cudaGetLastError();
+}
+
+}  // namespace tc
+}  // namespace confu
