@@ -46,6 +46,9 @@ struct SharedStorage {
     uint64_t s_full[2], p_full[2], o_done[2];
     uint32_t tmem_base;
     int abort;
+    // per softmax warp: a 32 x 32 fp32 tile for turning "one thread per row" into whole-line stores;
+    // the four floats (row, 4q .. 4q+3) sit at float4 index row * 8 + (q ^ (row & 7))
+    alignas(16) float4 xpose[8][32 * 8];
 };
 
 // ------------------------------------------------------------------------------------ PTX wrappers
@@ -510,42 +513,65 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
         // ---- epilogue of this pair / range ----
         if (!mbar_wait(&sh.o_done[t], seg & 1, &sh.abort)) return;
         tc_fence_after();
+        // O_t leaves tensor memory one row per thread; written like that, every store instruction of a
+        // warp would touch 32 different lines.  Each 32-column chunk goes through the warp's
+        // shared-memory tile instead and is stored in 16-byte pieces that cover whole rows: eight
+        // rows per instruction for the bf16 output (4 lanes x 16 B each), four for an fp32 partial.
         const int h = s.g * G + hl;
-        if (s.part_slot < 0) {
-            const float inv_l = 1.f / l;
-            __nv_bfloat16* orow = prm.out + (((size_t)s.b * R + r) * Hq + h) * kD;
+        const int lane = threadIdx.x & 31;
+        float4* xp = sh.xpose[threadIdx.x >> 5];
+        const bool whole = s.part_slot < 0;
+        const float inv_l = whole ? 1.f / l : 1.f;
+        // where this lane's pieces go: row 8 kk + lane / 4 of the warp's 32 (output), row 4 kk + lane / 8 (partial)
+        __nv_bfloat16* o_ptr[4];
+        float* p_ptr = nullptr;
+        if (whole) {
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                uint32_t ov[32];
-                tmem_ld32(o_addr + q4 * 32, ov);
-                tc_wait_ld();
-                if (row_valid) {
+            for (int kk = 0; kk < 4; ++kk) {
+                const int lr = warp_in_wg * 32 + 8 * kk + (lane >> 2);
+                const int rk = kGroupRows * s.rg + 32 * t + lr / G;
+                o_ptr[kk] = (lr < 32 * G && rk < R)
+                                ? prm.out + (((size_t)s.b * R + rk) * Hq + s.g * G + lr % G) * kD + 8 * (lane & 3)
+                                : nullptr;
+            }
+        } else {
+            p_ptr = prm.partials + (size_t)s.part_slot * (partial_slot_bytes() / sizeof(float)) +
+                    (size_t)(t * 128 + warp_in_wg * 32 + (lane >> 3)) * kPartD + 4 * (lane & 7);
+        }
+#pragma unroll 1
+        for (int q4 = 0; q4 < 4; ++q4) {
+            uint32_t ov[32];
+            tmem_ld32(o_addr + q4 * 32, ov);
+            tc_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 pkt;
-                        pkt.x = pack_bf16(__uint_as_float(ov[8 * j + 0]) * inv_l, __uint_as_float(ov[8 * j + 1]) * inv_l);
-                        pkt.y = pack_bf16(__uint_as_float(ov[8 * j + 2]) * inv_l, __uint_as_float(ov[8 * j + 3]) * inv_l);
-                        pkt.z = pack_bf16(__uint_as_float(ov[8 * j + 4]) * inv_l, __uint_as_float(ov[8 * j + 5]) * inv_l);
-                        pkt.w = pack_bf16(__uint_as_float(ov[8 * j + 6]) * inv_l, __uint_as_float(ov[8 * j + 7]) * inv_l);
-                        *reinterpret_cast<uint4*>(orow + q4 * 32 + j * 8) = pkt;
-                    }
+            for (int q = 0; q < 8; ++q)
+                xp[lane * 8 + (q ^ (lane & 7))] =
+                    make_float4(__uint_as_float(ov[4 * q]) * inv_l, __uint_as_float(ov[4 * q + 1]) * inv_l,
+                                __uint_as_float(ov[4 * q + 2]) * inv_l, __uint_as_float(ov[4 * q + 3]) * inv_l);
+            __syncwarp();
+            if (whole) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const int k = 8 * kk + (lane >> 2), q = 2 * (lane & 3);
+                    const float4 a = xp[k * 8 + (q ^ (k & 7))], c = xp[k * 8 + ((q + 1) ^ (k & 7))];
+                    if (o_ptr[kk])
+                        *reinterpret_cast<uint4*>(o_ptr[kk] + q4 * 32) =
+                            make_uint4(pack_bf16(a.x, a.y), pack_bf16(a.z, a.w), pack_bf16(c.x, c.y), pack_bf16(c.z, c.w));
+                }
+            } else {
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const int k = 4 * kk + (lane >> 3);
+                    *reinterpret_cast<float4*>(p_ptr + (size_t)(4 * kk) * kPartD + q4 * 32) = xp[k * 8 + ((lane & 7) ^ (k & 7))];
                 }
             }
+            __syncwarp();
+        }
+        if (whole) {
             if (row_valid && prm.lse)
                 prm.lse[((size_t)s.b * R + r) * Hq + h] = (m_ref + log2f(l)) * 0.6931471805599453f;
         } else {
-            float* slot = prm.partials + (size_t)s.part_slot * (partial_slot_bytes() / sizeof(float));
-            float* prow = slot + (size_t)(t * 128 + lane_row) * kPartD;
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                uint32_t ov[32];
-                tmem_ld32(o_addr + q4 * 32, ov);
-                tc_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    *reinterpret_cast<uint4*>(prow + q4 * 32 + j * 4) = make_uint4(ov[4 * j], ov[4 * j + 1], ov[4 * j + 2], ov[4 * j + 3]);
-            }
-            float* ml = slot + (size_t)kPartRows * kPartD;
+            float* ml = prm.partials + (size_t)s.part_slot * (partial_slot_bytes() / sizeof(float)) + (size_t)kPartRows * kPartD;
             ml[t * 128 + lane_row] = m_ref;
             ml[kPartRows + t * 128 + lane_row] = l;
         }
