@@ -589,6 +589,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 {
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& sh = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the kernels before this one have completed
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
     if ((int)blockIdx.x >= pv.hdr->n_ctas) return;
     const int warp = threadIdx.x >> 5;
@@ -726,8 +727,20 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    attention_tc_kernel<<<ctx->sm_count, kThreads, smem, st>>>(q_map, k_map, v_map, ks_map, vs_map, prm);
-    cudaError_t e = cudaGetLastError();
+    // Launched as a programmatic dependent of whatever precedes it in the stream: its CTAs may be
+    // scheduled while the predecessor drains; the kernel waits (griddepcontrol.wait, first thing) for
+    // the predecessor's completion and memory flush before it touches global memory.
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctx->sm_count);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attention_tc_kernel, q_map, k_map, v_map, ks_map, vs_map, prm);
     if (e != cudaSuccess) return e;
     return launch_combine(prm, ctx->sm_count, st);
 }

@@ -12,6 +12,7 @@ namespace tc {
 // 256-byte lines.
 __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the attention kernel has completed
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
     const int pair = blockIdx.x, t = blockIdx.y;
     // pairs: sequence major, then kv head, then row group
@@ -64,6 +65,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
 constexpr int kCombineRowsPerBlock = 16;
 __global__ void __launch_bounds__(32 * kCombineRowsPerBlock) combine_wide_kernel(const Params prm)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the attention kernel has completed
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
     const int pair = blockIdx.x, t = blockIdx.y;
     // pairs: sequence major, then kv head, then row group
@@ -133,11 +135,22 @@ cudaError_t launch_combine(const Params& prm, int sm_count, cudaStream_t st)
 {
     // few pairs for the machine (each spread over several CTAs): the merge that is parallel over parts
     const int n_pairs = prm.d.B * prm.d.Hkv * prm.n_rg;
-    if (sm_count >= 2 * n_pairs)
-        combine_wide_kernel<<<dim3(n_pairs, prm.n_mt, 128 / kCombineRowsPerBlock), 32 * kCombineRowsPerBlock, 0, st>>>(prm);
-    else
-        combine_kernel<<<dim3(n_pairs, prm.n_mt, 4), 256, 0, st>>>(prm);
-    return cudaGetLastError();
+    // a programmatic dependent of the attention kernel: scheduled while that one drains, waits at its top
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = st;
+    cfg.attrs = pdl;
+    cfg.numAttrs = 1;
+    if (sm_count >= 2 * n_pairs) {
+        cfg.gridDim = dim3((unsigned)n_pairs, (unsigned)prm.n_mt, 128 / kCombineRowsPerBlock);
+        cfg.blockDim = dim3(32 * kCombineRowsPerBlock);
+        return cudaLaunchKernelEx(&cfg, combine_wide_kernel, prm);
+    }
+    cfg.gridDim = dim3((unsigned)n_pairs, (unsigned)prm.n_mt, 4);
+    cfg.blockDim = dim3(256);
+    return cudaLaunchKernelEx(&cfg, combine_kernel, prm);
 }
 
 }  // namespace tc
