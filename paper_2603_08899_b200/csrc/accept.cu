@@ -602,15 +602,26 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
                 __syncthreads();
                 if (tid == 0) { sh.Mt = M[0]; sh.invZt = (float)(1.0 / Z[0]); sh.Md = M[1]; sh.invZd = (float)(1.0 / Z[1]); }
             }
+            if (!lazy && tid < 32) {
+                // chunk statistics of the node's two rows -> maximum and normaliser of each: lanes 0-15
+                // take the target row's chunks, lanes 16-31 the draft row's; maxima and the fp64 sum
+                // are reduced inside each half warp (a fixed order, the same in every CTA)
+                __syncwarp();
+                const int c = tid & 15;
+                const RowStat* st = (tid < 16 ? st_t : st_d) + (size_t)sh.cur * kStatChunksMax;
+                const float m = c < nch ? st[c].m : -INFINITY;
+                const float sc = c < nch ? st[c].s : 0.f;
+                float mm = m;
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
+                double z = m > -INFINITY ? (double)sc * exp(((double)m - (double)mm) * inv_temp) : 0.0;
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+                if (tid == 0) { sh.Mt = mm; sh.invZt = (float)(1.0 / z); }
+                if (tid == 16) { sh.Md = mm; sh.invZd = (float)(1.0 / z); }
+            }
             if (tid == 0) {
                 const int cur = sh.cur;
-                if (!lazy) {
-                    float M; double Z; int a;
-                    merge_row(st_t + (size_t)cur * kStatChunksMax, nch, inv_temp, M, Z, a);
-                    sh.Mt = M; sh.invZt = (float)(1.0 / Z);
-                    merge_row(st_d + (size_t)cur * kStatChunksMax, nch, inv_temp, M, Z, a);
-                    sh.Md = M; sh.invZd = (float)(1.0 / Z);
-                }
                 int n = 0;
                 for (int i = cur + 1; i < Tn; ++i) if (par[i] == cur) sh.ch[n++] = i;
                 sh.nch = n; sh.k = 0; sh.accepted = -1;
