@@ -49,6 +49,13 @@ CASES = {
     "bf16_rows_128_chain": _cfg(B=1, T=64, C=64, S=16, tree="chain", prefix=257, seed=52),
     "fp32_rows_100": _cfg(kv_dtype=torch.float32, T=50, C=50, prefix=(10, 150), max_depth=7, fanout=(1, 4), seed=53),
     "bf16_d64_rows_90": _cfg(D=64, T=45, C=45, prefix=(10, 150), max_depth=7, fanout=(1, 4), seed=54),
+    # the largest soft-prompt block the tensor-core path takes (one whole key tile), and a ragged one
+    "bf16_soft_128": _cfg(S=128, seed=55),
+    "bf16_soft_100": _cfg(S=100, T=20, C=20, seed=56),
+    # one pair of 131 key tiles: every CTA gets a single tile, the merge sees ~130 parts (more than one group of 32)
+    "bf16_one_pair_130_parts": _cfg(B=1, Hq=4, Hkv=1, prefix=16500, seed=57),
+    # more pairs than SMs: whole pairs per CTA, few splits
+    "bf16_many_short_sequences": _cfg(B=170, Hq=4, Hkv=2, prefix=(1, 260), seed=58),
 }
 
 
