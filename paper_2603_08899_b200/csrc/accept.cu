@@ -215,6 +215,7 @@ struct WalkShared {
     // maximum and sum of exponentials of two rows at once (statistics on demand)
     float red2_m[2][kWalkThreads / 32], red2_s[2][kWalkThreads / 32], cl2_m[2][kWalkCluster], cl2_s[2][kWalkCluster];
     int next;
+    int cnt0, cnt1, below[64];     // children scan of the walk
 };
 
 // merged statistics of one row from its chunk partials (fixed order)
@@ -235,9 +236,9 @@ __device__ inline void merge_row(const RowStat* st, int nch, double inv_temp, fl
 __device__ __forceinline__ float weight_at(float tx, float dx, int idx, int level, int mode, const WalkShared& sh,
                                            float k2)
 {
-    float p = exp2f((tx - sh.Mt) * k2) * sh.invZt;
+    float p = ex2((tx - sh.Mt) * k2) * sh.invZt;
     if (level == 0) return p;
-    float q = exp2f((dx - sh.Md) * k2) * sh.invZd;
+    float q = ex2((dx - sh.Md) * k2) * sh.invZd;
     for (int j = 0; j + 1 < level; ++j) {
         const float pn = fmaxf(p - q, 0.f) * sh.invZ[j];
         if (mode == 1) q = (idx == sh.xs[j]) ? 0.f : q * sh.cs[j];
@@ -246,8 +247,58 @@ __device__ __forceinline__ float weight_at(float tx, float dx, int idx, int leve
     return fmaxf(p - q, 0.f);
 }
 
-// Sum of weight_at(., level) over the vocabulary, strip by strip, in double; fills sh.strip[] of
-// every CTA of the cluster.  CTA `rank` computes strips rank, rank + kWalkCluster, ...
+// fp32 sums of the weights of two runs of eight entries, i0 .. i0 + 7 and i1 .. i1 + 7 (i1 < 0: none),
+// all loads issued before any weight is computed.  fp64 arithmetic is scarce on this part: everything
+// above a thread's eight is summed in fp64.  A real call on purpose: a pass over the vocabulary runs
+// its code once or twice, so what counts is how little code there is to fetch, and this body is the
+// same for every strip, pass and level.
+template <typename T>
+__device__ __noinline__ float2 weight_sum8x2(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok,
+                                             int i0, int i1, int level, int mode, const WalkShared& sh, float k2)
+{
+    float tx[2][kEpt], dx[2][kEpt];
+    load8(trow, i0, V, vec_ok, tx[0]);
+    if (level > 0) load8(drow, i0, V, vec_ok, dx[0]);
+    if (i1 >= 0) {
+        load8(trow, i1, V, vec_ok, tx[1]);
+        if (level > 0) load8(drow, i1, V, vec_ok, dx[1]);
+    }
+    float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < kEpt; ++j) acc.x += weight_at(tx[0][j], level > 0 ? dx[0][j] : 0.f, i0 + j, level, mode, sh, k2);
+    if (i1 >= 0) {
+#pragma unroll
+        for (int j = 0; j < kEpt; ++j) acc.y += weight_at(tx[1][j], level > 0 ? dx[1][j] : 0.f, i1 + j, level, mode, sh, k2);
+    }
+    return acc;
+}
+
+// Inverse-CDF search inside one run of eight entries: `run` is the fp64 sum of all weights before
+// entry i0.  Returns the first entry whose running sum exceeds the target (INT_MAX: none here);
+// last = the highest entry of the eight with a positive weight (-1: none).
+template <typename T>
+__device__ __noinline__ int find8(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok, int i0,
+                                  int level, int mode, const WalkShared& sh, float k2, double run, double target,
+                                  int& last)
+{
+    float tx[kEpt], dx[kEpt];
+    load8(trow, i0, V, vec_ok, tx);
+    if (level > 0) load8(drow, i0, V, vec_ok, dx);
+    int cand = INT_MAX;
+    last = -1;
+#pragma unroll
+    for (int j = 0; j < kEpt; ++j) {
+        const float w = weight_at(tx[j], level > 0 ? dx[j] : 0.f, i0 + j, level, mode, sh, k2);
+        run += (double)w;
+        if (w > 0.f) last = i0 + j;
+        if (cand == INT_MAX && run > target) cand = i0 + j;
+    }
+    return cand;
+}
+
+// Sum of weight_at(., level) over the vocabulary, strip by strip; fills sh.strip[] of every CTA of
+// the cluster and returns the total to thread 0 (0 to the others).  CTA `rank` computes strips
+// rank, rank + kWalkCluster, ...
 template <typename T>
 __device__ double full_pass(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok, int level,
                             int mode, WalkShared& sh, float k2)
@@ -256,28 +307,15 @@ __device__ double full_pass(const T* __restrict__ trow, const T* __restrict__ dr
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x, n_strips = (V + kStrip - 1) / kStrip;
-    for (int sa = rank; sa < n_strips; sa += 2 * kWalkCluster) {
-        float tx[2][kEpt], dx[2][kEpt];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int st = sa + u * kWalkCluster;
-            const int i0 = st * kStrip + tid * kEpt;
-            if (st < n_strips) {
-                load8(trow, i0, V, vec_ok, tx[u]);
-                if (level > 0) load8(drow, i0, V, vec_ok, dx[u]);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int st = sa + u * kWalkCluster;
-            if (st >= n_strips) break;
-            const int i0 = st * kStrip + tid * kEpt;
-            double acc = 0.0;
-#pragma unroll
-            for (int j = 0; j < kEpt; ++j)
-                acc += (double)weight_at(tx[u][j], level > 0 ? dx[u][j] : 0.f, i0 + j, level, mode, sh, k2);
-            acc = warp_sum(acc);
-            if ((tid & 31) == 0) sh.warp_part[st][tid >> 5] = acc;
+#pragma unroll 1
+    for (int st = rank; st < n_strips; st += 2 * kWalkCluster) {
+        const int st1 = st + kWalkCluster < n_strips ? st + kWalkCluster : -1;
+        const float2 a8 = weight_sum8x2(trow, drow, V, vec_ok, st * kStrip + tid * kEpt,
+                                        st1 >= 0 ? st1 * kStrip + tid * kEpt : -1, level, mode, sh, k2);
+        const double a0 = warp_sum((double)a8.x), a1 = warp_sum((double)a8.y);
+        if ((tid & 31) == 0) {
+            sh.warp_part[st][tid >> 5] = a0;
+            if (st1 >= 0) sh.warp_part[st1][tid >> 5] = a1;
         }
     }
     __syncthreads();
@@ -292,8 +330,9 @@ __device__ double full_pass(const T* __restrict__ trow, const T* __restrict__ dr
         }
     }
     cluster.sync();
-    double tot = 0.0;
-    for (int st = 0; st < n_strips; ++st) tot += sh.strip[st];
+    double tot = 0.0;                    // thread 0 alone needs the total
+    if (tid == 0)
+        for (int st = 0; st < n_strips; ++st) tot += sh.strip[st];
     return tot;
 }
 
@@ -324,16 +363,8 @@ __device__ int locate(const T* __restrict__ trow, const T* __restrict__ drow, in
     }
     __syncthreads();
     const int i0 = sh.strip_sel * kStrip + tid * kEpt;
-    float tx[kEpt], dx[kEpt];
-    load8(trow, i0, V, vec_ok, tx);
-    if (level > 0) load8(drow, i0, V, vec_ok, dx);
-    float w[kEpt];
-    double loc = 0.0;
-#pragma unroll
-    for (int j = 0; j < kEpt; ++j) {
-        w[j] = weight_at(tx[j], level > 0 ? dx[j] : 0.f, i0 + j, level, mode, sh, k2);
-        loc += (double)w[j];
-    }
+    // the thread's eight weights, summed as in full_pass
+    const double loc = (double)weight_sum8x2(trow, drow, V, vec_ok, i0, -1, level, mode, sh, k2).x;
     // block exclusive scan of loc (double): warp scan + warp totals
     double incl = loc;
 #pragma unroll
@@ -345,14 +376,9 @@ __device__ int locate(const T* __restrict__ trow, const T* __restrict__ drow, in
     __syncthreads();
     double off = sh.strip_off;
     for (int wi = 0; wi < (tid >> 5); ++wi) off += sh.scan[wi];
-    double run = off + (incl - loc);
-    int cand = INT_MAX, last = -1;
-#pragma unroll
-    for (int j = 0; j < kEpt; ++j) {
-        run += (double)w[j];
-        if (w[j] > 0.f) last = i0 + j;
-        if (cand == INT_MAX && run > sh.target) cand = i0 + j;
-    }
+    const double run = off + (incl - loc);
+    int last;
+    const int cand = find8(trow, drow, V, vec_ok, i0, level, mode, sh, k2, run, sh.target, last);
     if (cand != INT_MAX) atomicMin(&sh.pick, cand);
     if (last >= 0) atomicMax(&sh.pick_last, last);
     __syncthreads();
@@ -484,11 +510,15 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
             if (!greedy && mode == 1 && tid > 0)
                 for (int j = tid + 1; j < Tn; ++j)
                     if (par[j] == p && tok[j] == tok[tid]) code = CONFU_ST_DUP_SIBLING;
-            if (code == INT_MAX && !lazy)
-                for (int c = 0; c < nch; ++c)
-                    if (st_t[(size_t)tid * kStatChunksMax + c].flag ||
-                        (!greedy && st_d[(size_t)tid * kStatChunksMax + c].flag))
-                        code = CONFU_ST_NONFINITE;
+            if (code == INT_MAX && !lazy) {
+                // (all flags are fetched before any is looked at: independent loads, one round trip)
+                int f = 0;
+                for (int c = 0; c < nch; ++c) {
+                    f |= st_t[(size_t)tid * kStatChunksMax + c].flag;
+                    if (!greedy) f |= st_d[(size_t)tid * kStatChunksMax + c].flag;
+                }
+                if (f) code = CONFU_ST_NONFINITE;
+            }
         }
         if (code != INT_MAX) atomicMin(&sh.code, code);
     }
@@ -512,6 +542,7 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
     const float k2 = (float)inv_temp * kLog2e;
 
     if (tid == 0) { sh.cur = 0; sh.len = 0; sh.path[0] = 0; sh.tests = 0; sh.rejections = 0; sh.done = 0; }
+    __syncthreads();
 
     int lazy_code = 0;                // statistics on demand: a non-finite logit in a row that was needed
     if (greedy && lazy) {
@@ -620,12 +651,19 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
                 if (tid == 0) { sh.Mt = mm; sh.invZt = (float)(1.0 / z); }
                 if (tid == 16) { sh.Md = mm; sh.invZd = (float)(1.0 / z); }
             }
-            if (tid == 0) {
+            // children of the current node in increasing index: nodes 0-31 by the lanes of warp 0, 32-63
+            // by warp 1, each child's place = the children before it
+            if (tid < 2 * 32) {
                 const int cur = sh.cur;
-                int n = 0;
-                for (int i = cur + 1; i < Tn; ++i) if (par[i] == cur) sh.ch[n++] = i;
-                sh.nch = n; sh.k = 0; sh.accepted = -1;
+                const bool is_child = tid > cur && tid < Tn && par[tid] == cur;
+                const unsigned mask = __ballot_sync(0xffffffffu, is_child);
+                if (tid == 0) sh.cnt0 = __popc(mask);
+                if (tid == 32) sh.cnt1 = __popc(mask);
+                sh.below[tid] = __popc(mask & ((1u << (tid & 31)) - 1u)) | (is_child ? 0x100 : 0);
             }
+            __syncthreads();
+            if (tid < 2 * 32 && (sh.below[tid] & 0x100)) sh.ch[(sh.below[tid] & 0xff) + (tid >= 32 ? sh.cnt0 : 0)] = tid;
+            if (tid == 0) { sh.nch = sh.cnt0 + sh.cnt1; sh.k = 0; sh.accepted = -1; }
             __syncthreads();
             const int cur = sh.cur;
             const T* trow = tl + ((size_t)b * Tn + cur) * V;
