@@ -376,39 +376,48 @@ def run_ours(args, cfg):
         for l in range(cfg.L):
             h["krows"].append(step.k[l][idx].view(cfg.B, R, cfg.Hkv, cfg.D).cpu().pin_memory())
             h["vrows"].append(step.v[l][idx].view(cfg.B, R, cfg.Hkv, cfg.D).cpu().pin_memory())
-        d_krows = torch.empty_like(h["krows"][0], device=device)
-        d_vrows = torch.empty_like(h["vrows"][0], device=device)
+        d_krows = [torch.empty_like(t, device=device) for t in h["krows"]]     # per layer: copies run ahead of compute
+        d_vrows = [torch.empty_like(t, device=device) for t in h["vrows"]]
         res_host = {k: torch.empty_like(getattr(step, k), device="cpu").pin_memory()
                     for k in ("accept_len", "path", "next_token", "future_row", "new_prefix_len", "status")}
         h2d = sum(t.numel() * t.element_size() for t in h["q"] + h["krows"] + h["vrows"]) + \
             sum(h[k].numel() * h[k].element_size() for k in ("tl", "dl", "tok", "u", "parent", "owner"))
         d2h = sum(t.numel() * t.element_size() for t in res_host.values())
 
-        # The logits (the bulk of the bytes) travel on a second stream while the attention layers run;
-        # the acceptance call waits for them, and the next step's copy waits for this step's acceptance.
+        # All inputs of a step travel on one copy stream in the order the step uses them (tree arrays, then
+        # layer by layer Q and the rows' K/V, the logits last), each followed by an event the compute stream
+        # waits for; the copies of the next step start when this step's last kernel has been enqueued and
+        # finished (its inputs must not be overwritten under it).
         copy_stream = torch.cuda.Stream()
-        ev_logits, ev_accept = torch.cuda.Event(), torch.cuda.Event()
-        ev_accept.record()
+        ev_tree = torch.cuda.Event()
+        ev_layer = [torch.cuda.Event() for _ in range(cfg.L)]
+        ev_logits, ev_done = torch.cuda.Event(), torch.cuda.Event()
+        ev_done.record()
 
         def e2e_step():
             main = torch.cuda.current_stream()
-            copy_stream.wait_event(ev_accept)
+            copy_stream.wait_event(ev_done)
             with torch.cuda.stream(copy_stream):
+                step.parent.copy_(h["parent"], non_blocking=True)
+                if cfg.C:
+                    step.con_owner.copy_(h["owner"], non_blocking=True)
+                ev_tree.record(copy_stream)
+                for l in range(cfg.L):
+                    step.q[l].copy_(h["q"][l], non_blocking=True)
+                    d_krows[l].copy_(h["krows"][l], non_blocking=True)
+                    d_vrows[l].copy_(h["vrows"][l], non_blocking=True)
+                    ev_layer[l].record(copy_stream)
                 step.tl.copy_(h["tl"], non_blocking=True)
                 step.dl.copy_(h["dl"], non_blocking=True)
                 step.tokens.copy_(h["tok"], non_blocking=True)
                 step.uniforms.copy_(h["u"], non_blocking=True)
                 ev_logits.record(copy_stream)
-            step.parent.copy_(h["parent"], non_blocking=True)
-            if cfg.C:
-                step.con_owner.copy_(h["owner"], non_blocking=True)
+            main.wait_event(ev_tree)
             cb.confu_tree_plan(step.ctx, step.dims, step.seq_start, step.prefix_len, step.parent, step.con_owner,
                                step.plan, step.status)
             for l in range(cfg.L):
-                step.q[l].copy_(h["q"][l], non_blocking=True)
-                d_krows.copy_(h["krows"][l], non_blocking=True)
-                d_vrows.copy_(h["vrows"][l], non_blocking=True)
-                cb.confu_kv_append(step.ctx, step.dims, d_krows, d_vrows, step.k[l], step.v[l], step.seq_start,
+                main.wait_event(ev_layer[l])
+                cb.confu_kv_append(step.ctx, step.dims, d_krows[l], d_vrows[l], step.k[l], step.v[l], step.seq_start,
                                    step.prefix_len)
                 cb.confu_tree_attention(step.ctx, step.dims, step.q[l], step.k[l], step.v[l], step.n_slots,
                                         step.seq_start, step.prefix_len, step.ks[l] if step.ks else None,
@@ -416,8 +425,8 @@ def run_ours(args, cfg):
                                         step.status)
             main.wait_event(ev_logits)
             step.run_accept(1.0)
-            ev_accept.record(main)
             step.run_compact()
+            ev_done.record(main)
             for k, t in res_host.items():
                 t.copy_(getattr(step, k), non_blocking=True)
 
@@ -479,7 +488,7 @@ def run_ours(args, cfg):
             "value": e2e[0], "unit": UNIT, "h2d_bytes_per_step": e2e[3], "d2h_bytes_per_step": e2e[4],
             "ms_per_step": e2e[1], "steps": e2e[2],
             "note": "per step: Q, the R rows' K/V (all layers), both logit matrices, tree arrays and uniforms "
-                    "copied from pinned host memory (logits on a second stream, overlapping the attention layers); "
+                    "copied from pinned host memory on a copy stream that runs ahead of the compute stream (an event per layer); "
                     "results copied back; the prefix KV cache is resident state"},
         "gpu_launches": args.steps * step.launches_per_step(),
         "clocks": clocks,
