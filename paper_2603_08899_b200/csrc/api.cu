@@ -31,7 +31,7 @@ int cuda_fail(confu_ctx* ctx, cudaError_t e)
 
 // workspace carving: [plan built by the attention call itself][split-KV partial slots]
 size_t ws_plan_offset() { return 0; }
-size_t ws_partial_offset(const confu_dims* d) { return align_up(plan_bytes(d->B), 256); }
+size_t ws_partial_offset(const confu_dims* d) { return align_up(plan_bytes(d->B, d->Hkv), 256); }
 size_t ws_total(const confu_ctx* ctx, const confu_dims* d)
 {
     return ws_partial_offset(d) + (size_t)2 * ctx->sm_count * partial_slot_bytes();
@@ -132,7 +132,7 @@ const char* confu_last_cuda_error(const confu_ctx* ctx)
 size_t confu_plan_bytes(const confu_ctx* ctx, const confu_dims* dims)
 {
     if (!ctx || check_dims(dims) != CONFU_OK) return 0;
-    return plan_bytes(dims->B);
+    return plan_bytes(dims->B, dims->Hkv);
 }
 
 int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims, const int64_t* seq_start, const int32_t* prefix_len,

@@ -186,67 +186,40 @@ struct Segment {
     int part_slot;     // -1: the range covers the whole pair, write the output directly
 };
 
+// A CTA's runs of key tiles come from the plan: one 48-byte descriptor each, in walking order.
 struct Walker {
-    const PlanView pv;
-    int64_t f, f1;             // this CTA's share of the cost line: positions [f, f1)
-    int cta;
-    const Params& prm;
-    __device__ Walker(const PlanView& v, const Params& p, int cta_) : pv(v), cta(cta_), prm(p)
+    const SegDesc* cur;
+    const SegDesc* end;
+    bool soft;
+    __device__ Walker(const PlanView& v, const Params& p, int cta) : soft(p.d.S > 0)
     {
-        const int64_t N = v.hdr->n_tiles;
-        const int64_t n = v.hdr->n_ctas;
-        f = (int64_t)cta_ * N / n;
-        f1 = (int64_t)(cta_ + 1) * N / n;
+        cur = v.segs + v.seg_begin[cta];
+        end = v.segs + v.seg_begin[cta + 1];
     }
-    // Next non-empty run of key tiles of one pair inside the share; false when the share is used up.
+    // Next run of key tiles of one pair inside the share; false when the share is used up.
     __device__ bool next(Segment& s)
     {
-        while (f < f1) {
-            int lo = 0, hi = prm.d.B;                  // largest b with tile_base[b] <= f
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (pv.tile_base[mid] <= f) lo = mid; else hi = mid;
-            }
-            const int nt = pv.tiles[lo];
-            const int cost = nt + kPairOverheadTiles;
-            const int64_t local = f - pv.tile_base[lo];
-            const int pos = (int)(local % cost);
-            const int64_t room = f1 - f;
-            const int take = (int)((int64_t)(cost - pos) <= room ? cost - pos : room);
-            f += take;
-            const int t0 = pos > kPairOverheadTiles ? pos - kPairOverheadTiles : 0;
-            const int t1 = pos + take > kPairOverheadTiles ? pos + take - kPairOverheadTiles : 0;
-            if (t1 <= t0) continue;                    // the share ended inside this pair's overhead zone
-            s.b = lo;
-            s.nt = nt;
-            const int pair = (int)(local / cost);       // pairs of a sequence: kv head major, row group minor
-            s.g = pair / prm.n_rg;
-            s.rg = pair % prm.n_rg;
-            s.t0 = t0;
-            s.t1 = t1;
-            s.nkt = nt - (prm.d.S > 0 ? 1 : 0);
-            s.P = prm.prefix_len[lo];
-            s.slot0 = prm.map.block_table ? 0 : prm.map.seq_start[lo];
-            const bool whole = t0 == 0 && t1 == nt;
-            s.part_slot = whole ? -1 : 2 * cta + (t1 < nt ? 1 : 0);
-            return true;
-        }
-        return false;
+        if (cur >= end) return false;
+        const uint4* q = reinterpret_cast<const uint4*>(cur);
+        const uint4 w0 = __ldg(q), w1 = __ldg(q + 1), w2 = __ldg(q + 2);
+        s.b = (int)w0.x;
+        s.g = (int)(w0.y & 0xffffu);
+        s.rg = (int)(w0.y >> 16);
+        s.t0 = (int)w0.z;
+        s.t1 = (int)w0.w;
+        s.nt = (int)w1.x;
+        s.nkt = s.nt - (soft ? 1 : 0);
+        s.P = (int)w1.y;
+        s.part_slot = (int)w1.z;
+        s.slot0 = (int64_t)(((uint64_t)w2.y << 32) | w2.x);
+        ++cur;
+        return true;
     }
 };
 
 // ------------------------------------------------------------------------------------ roles
 // Key tiles of the CTA's share, all pairs together, are numbered g = 0..n-1 in walking order; stage
 // g of the ring carries V of tile g-1 and K of tile g (stage 0 has no V, stage n no K).
-__device__ int count_tiles(const Params& prm, const PlanView& pv)
-{
-    Walker w(pv, prm, blockIdx.x);
-    Segment s;
-    int n = 0;
-    while (w.next(s)) n += s.t1 - s.t0;
-    return n;
-}
-
 struct TileRef {                       // where a key tile's K and V come from
     int g, z;                          // kv head, first slot (row) of the tile
     bool soft;                         // the soft-prompt tile
@@ -256,8 +229,8 @@ __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanVi
                               const CUtensorMap* k_map, const CUtensorMap* v_map, const CUtensorMap* ks_map,
                               const CUtensorMap* vs_map)
 {
-    const int n_total = count_tiles(prm, pv);
     Walker w(pv, prm, blockIdx.x);
+    const int n_total = (int)(w.end - w.cur);                 // runs; every run has at least one tile
     Segment s;
     uint32_t stage = 0, seg = 0;       // running stage / pair counters
     const int R = prm.d.T + prm.d.C;

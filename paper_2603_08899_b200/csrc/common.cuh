@@ -24,6 +24,8 @@ constexpr int kTileKeys = 128;                  // keys per attention tile (tens
 //   int32  bad[B]             non-zero: malformed tree, sequence skipped
 //   int32  tiles[B]           key tiles of one (sequence, kv head) pair, soft-prompt tile included
 //   int64  tile_base[B + 1]   position of sequence b's first pair on the flat cost line (exclusive scan)
+//   int32  seg_begin[kPlanMaxCtas + 1]   CTA c of the tensor-core kernel walks segs[seg_begin[c] .. seg_begin[c+1])
+//   SegDesc segs[B * Hkv * 2 + kPlanMaxCtas]   the runs of key tiles, one pair at a time, of every CTA in walking order
 //
 // The split-KV work is balanced on a "cost line": every (sequence, kv head) pair takes
 // tiles + kPairOverheadTiles consecutive positions (the overhead stands for loading Q, draining
@@ -39,23 +41,40 @@ struct PlanHeader {
     int64_t n_tiles;           // length N of the cost line
 };
 
+// One run of key tiles of one pair inside a CTA's share of the cost line.
+constexpr int kPlanMaxCtas = 256;
+struct alignas(16) SegDesc {
+    int32_t b, g_rg;           // sequence; kv head | group of 64 query rows << 16
+    int32_t t0, t1;            // tiles [t0, t1) of the pair
+    int32_t nt, P;             // tiles of the pair (soft-prompt tile included); prefix length
+    int32_t part_slot;         // -1: the run covers the whole pair; else the CTA's partial slot
+    int32_t pad0;
+    int64_t slot0;             // packed pool: the sequence's first slot
+    int64_t pad1;
+};
+static_assert(sizeof(SegDesc) == 48, "SegDesc is read as three 16-byte words");
+
 struct PlanView {
     PlanHeader* hdr;
     uint64_t* mask;
     int32_t* bad;
     int32_t* tiles;
     int64_t* tile_base;
+    int32_t* seg_begin;
+    SegDesc* segs;
 };
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-__host__ __device__ inline size_t plan_bytes(int B)
+__host__ __device__ inline size_t plan_bytes(int B, int Hkv)
 {
     size_t n = align_up(sizeof(PlanHeader), 256);
     n += align_up((size_t)B * kMaxRows * sizeof(uint64_t), 256);
     n += align_up((size_t)B * sizeof(int32_t), 256);
     n += align_up((size_t)B * sizeof(int32_t), 256);
     n += align_up((size_t)(B + 1) * sizeof(int64_t), 256);
+    n += align_up((size_t)(kPlanMaxCtas + 1) * sizeof(int32_t), 256);
+    n += align_up(((size_t)B * Hkv * 2 + kPlanMaxCtas) * sizeof(SegDesc), 256);
     return n;
 }
 
@@ -67,7 +86,9 @@ __host__ __device__ inline PlanView plan_view(void* base, int B)
     v.mask = (uint64_t*)p;                   p += align_up((size_t)B * kMaxRows * sizeof(uint64_t), 256);
     v.bad = (int32_t*)p;                     p += align_up((size_t)B * sizeof(int32_t), 256);
     v.tiles = (int32_t*)p;                   p += align_up((size_t)B * sizeof(int32_t), 256);
-    v.tile_base = (int64_t*)p;
+    v.tile_base = (int64_t*)p;               p += align_up((size_t)(B + 1) * sizeof(int64_t), 256);
+    v.seg_begin = (int32_t*)p;               p += align_up((size_t)(kPlanMaxCtas + 1) * sizeof(int32_t), 256);
+    v.segs = (SegDesc*)p;
     return v;
 }
 

@@ -64,6 +64,7 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
         }
         __syncthreads();
     }
+    __shared__ int s_count[kPlanMaxCtas + 1];
     if (threadIdx.x == 0) {
         int64_t acc = 0;
         for (int b = 0; b < B; ++b) {
@@ -76,10 +77,65 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
         h.B = B; h.Hkv = d.Hkv; h.T = T; h.C = C; h.S = d.S; h.R = R;
         h.n_tiles = acc;
         h.n_ctas = (int)(acc < (int64_t)sm_count ? acc : (int64_t)sm_count);
+        if (h.n_ctas > kPlanMaxCtas) h.n_ctas = kPlanMaxCtas;
         h.pad = 0;
         *pv.hdr = h;
     }
-    (void)seq_start;
+    __syncthreads();
+    // The runs of key tiles of every CTA of the tensor-core attention kernel, worked out once per step
+    // instead of by every role of every CTA of every layer: thread c walks CTA c's share of the cost
+    // line, first to count its runs, then (behind a prefix sum) to write them down.
+    const int n_rg = (R + kGroupRows - 1) / kGroupRows;
+    const int64_t N = pv.hdr->n_tiles;
+    const int n_ctas = pv.hdr->n_ctas;
+    for (int pass = 0; pass < 2; ++pass) {
+        const int c = threadIdx.x;
+        if (c < n_ctas) {
+            int64_t f = (int64_t)c * N / n_ctas;
+            const int64_t f1 = (int64_t)(c + 1) * N / n_ctas;
+            int n = 0;
+            SegDesc* out = pv.segs + (pass ? s_count[c] : 0);
+            int lo = 0;
+            while (f < f1) {
+                while (lo + 1 < B && pv.tile_base[lo + 1] <= f) ++lo;         // the sequence position f falls into
+                const int nt = pv.tiles[lo];
+                const int cost = nt + kPairOverheadTiles;
+                const int64_t local = f - pv.tile_base[lo];
+                const int pos = (int)(local % cost);
+                const int64_t room = f1 - f;
+                const int take = (int)((int64_t)(cost - pos) <= room ? cost - pos : room);
+                f += take;
+                const int t0 = pos > kPairOverheadTiles ? pos - kPairOverheadTiles : 0;
+                const int t1 = pos + take > kPairOverheadTiles ? pos + take - kPairOverheadTiles : 0;
+                if (t1 <= t0) continue;                    // the share ended inside this pair's overhead zone
+                if (pass) {
+                    const int pair = (int)(local / cost);       // pairs of a sequence: kv head major, row group minor
+                    SegDesc d;
+                    d.b = lo;
+                    d.g_rg = (pair / n_rg) | ((pair % n_rg) << 16);
+                    d.t0 = t0;
+                    d.t1 = t1;
+                    d.nt = nt;
+                    d.P = prefix_len[lo];
+                    d.part_slot = (t0 == 0 && t1 == nt) ? -1 : 2 * c + (t1 < nt ? 1 : 0);
+                    d.pad0 = 0;
+                    d.slot0 = seq_start ? seq_start[lo] : 0;
+                    d.pad1 = 0;
+                    out[n] = d;
+                }
+                ++n;
+            }
+            if (!pass) s_count[c] = n;
+        }
+        __syncthreads();
+        if (!pass && threadIdx.x == 0) {
+            int acc = 0;
+            for (int c2 = 0; c2 < n_ctas; ++c2) { const int n = s_count[c2]; s_count[c2] = acc; acc += n; }
+            s_count[n_ctas] = acc;
+            for (int c2 = 0; c2 <= n_ctas; ++c2) pv.seg_begin[c2] = s_count[c2];
+        }
+        __syncthreads();
+    }
 }
 
 cudaError_t launch_plan(const Ctx* ctx, const confu_dims& d, const int64_t* seq_start, const int32_t* prefix_len,
