@@ -147,7 +147,11 @@ int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims,
  * con_owner are read; otherwise they may be NULL).  Accumulation is fp32; bf16
  * inputs use the tensor-core path when D == 128 and Hq/Hkv <= 4; it takes the
  * query rows in groups of 64, so R > 64 streams the keys twice.
- * Needs the workspace.  All pointers device.
+ * Needs the workspace.  All pointers device.  Ordinary stream order holds: the kernels are
+ * launched as programmatic dependents (their blocks may be scheduled while the kernel before them
+ * drains) but wait for all earlier work of the stream before their first global memory access,
+ * and whatever is enqueued after the call sees completed results.  The call may be captured
+ * into a CUDA graph (no allocation, no synchronisation; call it once outside the capture first).
  */
 int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims,
                          const void* q, const void* k_cache, const void* v_cache, int64_t n_slots,
