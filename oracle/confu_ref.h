@@ -13,7 +13,11 @@
  * identical draft/target == always accept, hand-computed two-token cases,
  * textbook linear speculative sampling on a chain, exact-rational resampling,
  * and a chi-square test of the emitted-token marginal against the target
- * distribution (with a power check on a deliberately broken variant).
+ * distribution (with a power check on a deliberately broken variant).  The
+ * closeness records of the acceptance walks (ratio_margin, resample_margin,
+ * draw_margin, alt_token and the two "within 1e-5" counters) are pinned by
+ * hand-computed cases, by cases planted inside and just outside the 1e-5 band,
+ * and by exact-rational walks.
  * The whole verify step on synthetic inputs has no published numbers:
  * beyond those pins, end-to-end parity is unpinned.
  *

@@ -40,6 +40,12 @@ def test_hand_computed_cases(case):
     assert o["next_token"].tolist() == [case["next_token"]]
     assert o["future_row"].tolist() == [case["future_row"]]
     assert o["counters"][0, :2].tolist() == [case["tests"], case["rejections"]]
+    # how close each decision was: the record that decides whether a differing decision of another
+    # implementation is a rounding-limited one
+    assert o["ratio_margin"].item() == pytest.approx(case["ratio_margin"], abs=1e-12)
+    assert o["resample_margin"].item() == pytest.approx(case["resample_margin"], abs=1e-12)
+    assert o["alt_token"][0].tolist() == case["alt"]
+    assert o["counters"][0, 2:].tolist() == case["borderline"]
 
 
 def _random_case(T=12, V=50, B=4, seed=3, draft="independent", tree="random", C=3, dtype=torch.float32):
@@ -108,7 +114,8 @@ def test_resample_against_exact_rationals():
     """Residual and inverse CDF in exact rational arithmetic on a 12-token vocabulary."""
     rng = np.random.default_rng(7)
     V = 12
-    for trial in range(40):
+    n_checked = n_zero_neighbours = 0
+    for trial in range(80):
         pi = rng.integers(0, 9, V)
         qi = rng.integers(1, 9, V)
         pi[rng.integers(V)] += 1
@@ -138,6 +145,74 @@ def test_resample_against_exact_rationals():
                             torch.tensor([[float(u0), u1]], dtype=torch.float64))
         assert o["accept_len"].tolist() == [0]
         assert o["next_token"].tolist() == [want], (trial, want)
+        # the margins and the neighbouring tokens, in exact rationals as well
+        assert o["ratio_margin"].item() == pytest.approx(float(abs(ratio - Fraction(u1))), abs=1e-12)
+        lo = sum(res[:want], Fraction(0)) / tot
+        hi = lo + res[want] / tot
+        assert o["resample_margin"].item() == pytest.approx(float(min(u0 - lo, hi - u0)), abs=1e-12)
+        below = [k for k in range(want) if res[k] > 0]
+        above = [k for k in range(want + 1, V) if res[k] > 0]
+        assert o["alt_token"][0].tolist() == [below[-1] if below else -1, above[0] if above else -1]
+        n_checked += 1
+        n_zero_neighbours += (want > 0 and res[want - 1] == 0) or (want + 1 < V and res[want + 1] == 0)
+    assert n_checked >= 30 and n_zero_neighbours >= 5     # alt_token had zero-weight tokens to skip
+
+
+def test_ratio_margin_is_the_smallest_over_all_tests_made():
+    """Every ratio test of a walk in exact rationals (one level: three children, drawn without
+    replacement, all rejected or one accepted): the margin reported is the minimum over the tests
+    actually made, and the 1e-5 counter counts exactly those below the band."""
+    rng = np.random.default_rng(17)
+    V = 9
+    seen_accept = seen_all_rejected = 0
+    for trial in range(60):
+        pi, qi = rng.integers(1, 9, V), rng.integers(1, 9, V)
+        p = [Fraction(int(a), int(pi.sum())) for a in pi]
+        q = [Fraction(int(a), int(qi.sum())) for a in qi]
+        toks = [int(t) for t in rng.choice(V, 3, replace=False)]
+        us = [Fraction(int(rng.integers(3 << 14, 1 << 16)), 1 << 16) for _ in range(4)]   # high: rejections are common
+        if trial % 5 == 0:                                 # plant a test inside the band on the first child
+            us[1] = p[toks[0]] / q[toks[0]] + Fraction(3, 1000000)
+            if us[1] >= 1:
+                continue
+        pp, qq, margins, accepted, z = list(p), list(q), [], None, 1
+        for i, x in enumerate(toks):
+            ratio = pp[x] / qq[x]
+            margins.append(abs(ratio - us[1 + i]))
+            if us[1 + i] < ratio:
+                accepted = i
+                break
+            pp = [max(a - b, Fraction(0)) for a, b in zip(pp, qq)]
+            z = sum(pp)
+            if z == 0:
+                break
+            pp = [a / z for a in pp]
+            qq[x] = Fraction(0)
+            zq = sum(qq)
+            qq = [a / zq for a in qq]
+        if z == 0 or min(margins) < Fraction(1, 10**9) and trial % 5:
+            continue
+        rows_p = [[float(a) for a in p]] * 4
+        rows_q = [[float(a) for a in q]] * 4
+        o = ref.tree_accept(_logits_of(rows_p)[None], _logits_of(rows_q)[None], torch.tensor([[0] + toks]),
+                            torch.tensor([[-1, 0, 0, 0]]), None,
+                            torch.tensor([[float(u) for u in us]], dtype=torch.float64))
+        assert o["counters"][0, 0].item() == len(margins)
+        assert o["accept_len"].item() == (0 if accepted is None else 1)
+        assert o["ratio_margin"].item() == pytest.approx(float(min(margins)), abs=1e-12)
+        assert o["counters"][0, 2].item() == sum(float(m) < 1e-5 for m in margins)
+        seen_accept += accepted is not None
+        seen_all_rejected += accepted is None
+    assert seen_accept >= 10 and seen_all_rejected >= 10
+
+
+def test_no_ratio_test_means_infinite_margin():
+    # a single-node tree: no child to test, the bonus token comes straight from the root's row
+    o = ref.tree_accept(_logits_of([[0.25, 0.75]])[None], _logits_of([[0.5, 0.5]])[None], torch.tensor([[0]]),
+                        torch.tensor([[-1]]), None, torch.tensor([[0.5]], dtype=torch.float64))
+    assert math.isinf(o["ratio_margin"].item()) and o["counters"][0].tolist() == [0, 0, 0, 0]
+    assert o["next_token"].tolist() == [1] and o["resample_margin"].item() == pytest.approx(0.25, abs=1e-12)
+    assert o["alt_token"][0].tolist() == [0, -1]
 
 
 def test_greedy_equals_bruteforce_longest_matching_path():
@@ -291,7 +366,7 @@ def _emitted(o, tok):
     return first, second
 
 
-N_TRIALS = 60000
+N_TRIALS = 200000
 
 
 @pytest.mark.parametrize("mode", [1, 0])

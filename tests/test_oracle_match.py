@@ -3,7 +3,10 @@ other than itself: a hand-computed walk, the greedy walk it must reduce to at te
 numpy walk built on cumsum / searchsorted, the closed forms "every emitted token follows the
 target distribution" and "the root's draft is accepted with probability sum_x p(x) over its
 children's tokens", and the rule that only rows on the walked path are read."""
+from fractions import Fraction
+
 import numpy as np
+import pytest
 import torch
 from scipy import stats
 
@@ -33,10 +36,58 @@ def test_hand_computed_walk():
     assert o["next_token"].tolist() == [3]
     assert o["future_row"].tolist() == [4]               # node 3 has none: nearest ancestor that has is node 2
     assert o["counters"][0, :2].tolist() == [3, 2]
+    # how close the draws came to an edge of their cells: .65 in [.6, 1) -> .05; .4 in [0, .5) -> .1;
+    # .8 in [.75, 1) -> .05.  Smallest .05, none inside the 1e-5 band; around the last drawn token 3 of
+    # the uniform row: token 2 below, nothing above.
+    assert o["draw_margin"].item() == pytest.approx(0.05, abs=1e-12)
+    assert o["counters"][0, 2:].tolist() == [0, 0] and o["alt_token"][0].tolist() == [2, -1]
     # the first draw misses every child: nothing accepted, the drawn token itself is emitted
     u2 = torch.tensor([[.05, .99, .4, .8]], dtype=torch.float64)
     o2 = ref.tree_accept_match(tl, tokens, parent, owner, u2, temperature=1.0)
     assert o2["accept_len"].tolist() == [0] and o2["next_token"].tolist() == [0] and o2["future_row"].tolist() == [5]
+    assert o2["draw_margin"].item() == pytest.approx(0.05, abs=1e-12) and o2["alt_token"][0].tolist() == [-1, 1]
+    # a draw 2e-6 above the edge .6 of the root's row: still token 3 = node 2, counted as borderline
+    u3 = torch.tensor([[.600002, .99, .4, .8]], dtype=torch.float64)
+    o3 = ref.tree_accept_match(tl, tokens, parent, owner, u3, temperature=1.0)
+    assert o3["path"][0, :3].tolist() == [0, 2, 3] and o3["counters"][0].tolist() == [3, 2, 1, 0]
+    assert o3["draw_margin"].item() == pytest.approx(2e-6, abs=1e-12)
+
+
+def test_draw_margin_against_exact_rationals():
+    """A star tree with rational target rows: every draw of the walk redone in exact arithmetic; the
+    reported margin is the smallest distance of a draw to an edge of its cell."""
+    rng = np.random.default_rng(3)
+    V = 10
+    n_two_draws = 0
+    for trial in range(50):
+        rows = []
+        for _ in range(4):
+            w = rng.integers(0, 7, V)
+            w[rng.integers(V)] += 1
+            rows.append([Fraction(int(a), int(w.sum())) for a in w])
+        kids = [int(t) for t in rng.choice(V, 3, replace=False)]
+        us = [Fraction(int(rng.integers(0, 1 << 16)), 1 << 16) + Fraction(1, 1 << 20) for _ in range(4)]
+        cur, margins = 0, []
+        while True:
+            c, x = Fraction(0), None
+            for k in range(V):
+                lo, c = c, c + rows[cur][k]
+                if c > us[cur]:
+                    x = k
+                    break
+            margins.append(min(us[cur] - lo, c - us[cur]))
+            if cur == 0 and x in kids:
+                cur = 1 + kids.index(x)
+                continue
+            break
+        tl = _logits_of([[float(a) for a in r] for r in rows])[None]
+        o = ref.tree_accept_match(tl, torch.tensor([[0] + kids]), torch.tensor([[-1, 0, 0, 0]]), None,
+                                  torch.tensor([[float(u) for u in us]], dtype=torch.float64), temperature=1.0)
+        assert o["accept_len"].item() == (1 if cur else 0) and o["next_token"].item() == x
+        assert o["counters"][0, 0].item() == len(margins)
+        assert o["draw_margin"].item() == pytest.approx(float(min(margins)), abs=1e-12)
+        n_two_draws += len(margins) == 2
+    assert n_two_draws >= 8
 
 
 def _random_case(T=14, V=40, B=6, seed=11, dtype=torch.float32, sigma=2.0, tree="random"):
