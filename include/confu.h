@@ -20,7 +20,8 @@
  *     aligned; the caller owns every buffer it passes, for the whole time the
  *     enqueued work runs;
  *   - work is enqueued on the given stream (a cudaStream_t passed as void*); no call
- *     synchronises the host with the device and none allocates device memory;
+ *     synchronises the host with the device and none allocates device memory; the
+ *     context's device must be the current device of the calling thread;
  *   - data-dependent problems (a malformed tree, an out-of-range token, a
  *     non-finite logit, a bounded device-side wait that ran out) never trap: the
  *     kernels write a positive code into status[b] (int32, device, one per sequence).
@@ -34,6 +35,9 @@
  *   A layer's cache pool is [n_slots][Hkv][D]; sequence b owns slots
  *   seq_start[b] .. seq_start[b] + prefix_len[b] + R - 1: its prefix, then the K/V of
  *   its R query rows (written there by the caller before confu_tree_attention).
+ *   Slots that belong to no sequence, or lie past a sequence's last row (pool padding, the
+ *   unused tail of a page), are never interpreted: they may hold anything, NaN bit patterns
+ *   included, and need not be initialised.
  */
 #ifndef CONFU_H
 #define CONFU_H
@@ -68,7 +72,9 @@ enum {
     CONFU_ST_NONFINITE = 5,
     CONFU_ST_TIMEOUT = 6,        /* a bounded wait inside a kernel gave up */
     CONFU_ST_DEGENERATE = 7,     /* residual distribution had no mass; target row used instead */
-    CONFU_ST_TOO_DEEP = 8        /* accepted path longer than CONFU_MAX_DEPTH */
+    CONFU_ST_TOO_DEEP = 8,       /* accepted path longer than CONFU_MAX_DEPTH */
+    CONFU_ST_BAD_PATH = 9,       /* confu_kv_compact: path is not 0 = path[0] < path[1] < ... < T, or accept_len out of range */
+    CONFU_ST_BAD_PLAN = 10       /* confu_tree_attention: the plan was built for another attention path */
 };
 
 enum { CONFU_BF16 = 0, CONFU_F32 = 1 };
@@ -114,6 +120,33 @@ int confu_set_workspace(confu_ctx* ctx, void* device_ptr, size_t bytes);
  */
 int confu_set_paging(confu_ctx* ctx, const int32_t* block_table, int32_t max_pages);
 
+/*
+ * Options of a context (host state; they apply to the calls made after the setting).
+ *   CONFU_OPT_ATTENTION_PATH  which kernel confu_tree_plan prepares for and confu_tree_attention
+ *                             launches: CONFU_ATTENTION_AUTO (default: the fastest path that
+ *                             supports the dims), _GENERIC (CUDA cores, every dtype and shape),
+ *                             _TENSOR (tcgen05, one CTA per SM; bf16, D = 128, Hq/Hkv <= 4),
+ *                             _TENSOR_PAIR (tcgen05 two-SM instructions, one CTA pair per two SMs;
+ *                             as _TENSOR, and more than 32 query rows).  A path that does not
+ *                             support the dims makes the calls return CONFU_ERR_UNSUPPORTED.  Set
+ *                             it before confu_tree_plan: a plan only fits the path it was built
+ *                             for (status CONFU_ST_BAD_PLAN otherwise).
+ *   CONFU_OPT_WAIT_LIMIT_NS   wall-clock limit of every wait on a barrier inside the tensor-core
+ *                             kernels (default 2 s; 1 us .. 10 s).  A wait that runs out makes the
+ *                             kernel release what it holds and report CONFU_ST_TIMEOUT.
+ */
+enum { CONFU_OPT_ATTENTION_PATH = 1, CONFU_OPT_WAIT_LIMIT_NS = 2 };
+enum { CONFU_ATTENTION_AUTO = 0, CONFU_ATTENTION_GENERIC = 1, CONFU_ATTENTION_TENSOR = 2, CONFU_ATTENTION_TENSOR_PAIR = 3 };
+int confu_set_option(confu_ctx* ctx, int32_t option, int64_t value);
+
+/*
+ * Self-test of the bounded device-side wait (no counterpart in the paper): one warp waits, through
+ * the same routine the attention kernels use, on a barrier that nothing arrives at; after limit_ns
+ * (1 us .. 1 s) of wall clock the wait gives up and the kernel writes CONFU_ST_TIMEOUT to status[0]
+ * (device int32) and returns.  The context stays usable.
+ */
+int confu_selftest_bounded_wait(confu_ctx* ctx, int64_t limit_ns, int32_t* status, void* stream);
+
 const char* confu_status_string(int code);      /* host return codes and device status codes */
 const char* confu_last_cuda_error(const confu_ctx* ctx);
 
@@ -150,7 +183,8 @@ int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims,
  * Needs the workspace.  All pointers device.  Ordinary stream order holds: the kernels are
  * launched as programmatic dependents (their blocks may be scheduled while the kernel before them
  * drains) but wait for all earlier work of the stream before their first global memory access,
- * and whatever is enqueued after the call sees completed results.  The call may be captured
+ * and whatever is enqueued after the call sees completed results.  A sequence with a malformed tree
+ * (status 1 or 2) gets all-zero output rows and lse 0.  The call may be captured
  * into a CUDA graph (no allocation, no synchronisation; call it once outside the capture first).
  */
 int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims,
@@ -185,7 +219,10 @@ size_t confu_accept_workspace_bytes(int32_t B, int32_t T, int32_t V);
  * [B][CONFU_MAX_DEPTH+1] node ids root first, -1 padded; next_token [B];
  * future_row [B] = row index in [T,T+C) of the contemplate row owned by the last
  * accepted node, else by its nearest ancestor that has one, else -1; counters
- * (optional) [B][4] = ratio tests, rejections, reserved, reserved.
+ * (optional) [B][4] = ratio tests made, rejections, ratio tests with |p(x)/q(x) - u| < 1e-5,
+ * final draws (0 or 1) whose uniform lies within 1e-5 of an edge of the emitted token's cell
+ * of the normalised CDF.  The last two count the decisions that rounding could turn: an
+ * implementation in other arithmetic may legitimately differ there (greedy: always 0).
  * workspace: confu_accept_workspace_bytes().  All pointers device.
  * By default one streaming pass takes the softmax statistics of all T rows of both matrices
  * first, and a non-finite logit anywhere in them is an error (status 5).  With
@@ -238,7 +275,8 @@ int confu_tree_accept_static(int32_t B, int32_t T, int32_t C, int32_t V, int32_t
  * ((accept_len + 1) * V logits per sequence) and a non-finite logit is an error (status 5) only
  * there.  No draft logits, no workspace.
  * Outputs as for confu_tree_accept; counters (optional) [B][4] = draws, accepted nodes,
- * reserved, reserved.  All pointers device.
+ * draws within 1e-5 of an edge of the drawn token's cell of the normalised CDF, 0.  All pointers
+ * device.
  */
 int confu_tree_accept_match(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int32_t V, int32_t logit_dtype,
                             const void* target_logits, const int32_t* tokens, const int32_t* parent,
@@ -254,7 +292,11 @@ int confu_tree_accept_match(confu_ctx* ctx, int32_t B, int32_t T, int32_t C, int
  * (P_b = prefix_len[b]; slot P_b, the root, and the prefix stay), and
  * new_prefix_len[b] = P_b + accept_len[b] + 1.  Slots past the new prefix keep
  * unspecified contents.  k_cache_layers / v_cache_layers: DEVICE arrays of
- * n_layers device pointers.  Uses dims->Hkv, D, kv_dtype, B.  All pointers device.
+ * n_layers device pointers.  Uses dims->Hkv, D, kv_dtype, B, T.  All pointers device.
+ * The path is checked on the device before anything moves: 0 <= accept_len[b] <=
+ * CONFU_MAX_DEPTH and 0 = path[b][0] < path[b][1] < ... < path[b][accept_len[b]] < T (what
+ * confu_tree_accept writes; node ids grow along a root path).  Otherwise status[b] =
+ * CONFU_ST_BAD_PATH, nothing of sequence b is copied and new_prefix_len[b] = P_b + 1.
  */
 int confu_kv_compact(confu_ctx* ctx, const confu_dims* dims, int32_t n_layers,
                      void* const* k_cache_layers, void* const* v_cache_layers,
@@ -288,12 +330,15 @@ int confu_kv_append(confu_ctx* ctx, const confu_dims* dims, const void* k_rows, 
  * neither n_expert nor k_expert: both are arguments; limits n_expert <= 1024, k_expert <= 32).
  * All five tensors have the type `dtype` (CONFU_BF16 | CONFU_F32), rows contiguous; accumulation
  * is fp32.  Optional outputs: sel [B][k_expert] int32 (largest score first) and gate [B][k_expert]
- * fp32 (the weights used).  All pointers device, 16-byte aligned.
+ * fp32 (the weights used).  A sequence with a non-finite router logit (NaN or infinity in its
+ * hidden state, or in the router) gets status[b] = CONFU_ST_NONFINITE (status: optional device
+ * int32 [B]), an all-zero output row, sel = 0..k_expert-1 and gate = 0.  All pointers device,
+ * 16-byte aligned.
  */
 int confu_con_embedding(confu_ctx* ctx, int32_t B, int32_t H_in, int32_t H_out, int32_t n_expert, int32_t k_expert,
                         int32_t dtype, const void* hidden, const void* router_w, const void* router_b,
                         const void* experts, int32_t renormalize, void* out, int32_t* sel, float* gate,
-                        void* stream);
+                        int32_t* status, void* stream);
 
 #ifdef __cplusplus
 }

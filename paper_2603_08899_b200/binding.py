@@ -18,13 +18,16 @@ MAX_DEPTH = 63
 ACCEPT_LAZY = 0x100          # or-ed into sibling_mode: row statistics on demand
 BF16, F32 = 0, 1
 OK = 0
+OPT_ATTENTION_PATH, OPT_WAIT_LIMIT_NS = 1, 2
+ATTENTION_AUTO, ATTENTION_GENERIC, ATTENTION_TENSOR, ATTENTION_TENSOR_PAIR = 0, 1, 2, 3
+ST_TIMEOUT, ST_BAD_PATH, ST_BAD_PLAN = 6, 9, 10
 
 EXPORTS = [
     "confu_create", "confu_destroy", "confu_workspace_bytes", "confu_set_workspace", "confu_status_string",
     "confu_last_cuda_error", "confu_plan_bytes", "confu_tree_plan", "confu_tree_attention",
     "confu_accept_workspace_bytes", "confu_tree_accept", "confu_kv_compact", "confu_kv_append",
     "confu_tree_accept_static_max_rows", "confu_tree_accept_static", "confu_set_paging",
-    "confu_tree_accept_match", "confu_con_embedding",
+    "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_selftest_bounded_wait",
 ]
 
 
@@ -52,7 +55,7 @@ def lib():
         L.confu_last_cuda_error.restype = C.c_char_p
         for n in ("confu_create", "confu_destroy", "confu_set_workspace", "confu_tree_plan", "confu_tree_attention",
                   "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static", "confu_set_paging",
-                  "confu_tree_accept_match", "confu_con_embedding"):
+                  "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_selftest_bounded_wait"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -118,6 +121,15 @@ def confu_set_paging(ctx, block_table, max_pages=0):
     _check("confu_set_paging", lib().confu_set_paging(ctx, _ptr(block_table), C.c_int32(max_pages)))
 
 
+def confu_set_option(ctx, option, value):
+    _check("confu_set_option", lib().confu_set_option(ctx, C.c_int32(option), C.c_int64(value)))
+
+
+def confu_selftest_bounded_wait(ctx, limit_ns, status, stream=None):
+    _check("confu_selftest_bounded_wait",
+           lib().confu_selftest_bounded_wait(ctx, C.c_int64(limit_ns), _ptr(status), _stream(stream)), ctx)
+
+
 def confu_plan_bytes(ctx, dims):
     return int(lib().confu_plan_bytes(ctx, C.byref(dims)))
 
@@ -166,7 +178,7 @@ def confu_tree_accept_match(ctx, B, T, Cn, V, logit_dtype, target_logits, tokens
 
 
 def confu_con_embedding(ctx, hidden, router_w, router_b, experts, k_expert, renormalize, out, sel=None, gate=None,
-                        stream=None):
+                        status=None, stream=None):
     """Contemplate-token embedding: router -> softmax -> top-k experts -> weighted sum of their embeddings."""
     B, H_in = hidden.shape
     n_expert, H_out = experts.shape
@@ -174,7 +186,7 @@ def confu_con_embedding(ctx, hidden, router_w, router_b, experts, k_expert, reno
            lib().confu_con_embedding(ctx, C.c_int32(B), C.c_int32(H_in), C.c_int32(H_out), C.c_int32(n_expert),
                                      C.c_int32(k_expert), C.c_int32(dtype_code(hidden.dtype)), _ptr(hidden),
                                      _ptr(router_w), _ptr(router_b), _ptr(experts), C.c_int32(1 if renormalize else 0),
-                                     _ptr(out), _ptr(sel), _ptr(gate), _stream(stream)), ctx)
+                                     _ptr(out), _ptr(sel), _ptr(gate), _ptr(status), _stream(stream)), ctx)
 
 
 def confu_tree_accept_static_max_rows():

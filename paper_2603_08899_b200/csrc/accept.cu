@@ -216,7 +216,12 @@ struct WalkShared {
     float red2_m[2][kWalkThreads / 32], red2_s[2][kWalkThreads / 32], cl2_m[2][kWalkCluster], cl2_s[2][kWalkCluster];
     int next;
     int cnt0, cnt1, below[64];     // children scan of the walk
+    // closeness records: ratio tests (match rule: draws) within kBorderline of their threshold; the
+    // last inverse-CDF draw: sum of all weights, running sums before and behind the chosen entry
+    int border_tests, border_draw;
+    double total, pick_lo, pick_hi;
 };
+constexpr double kBorderline = 1e-5;
 
 // merged statistics of one row from its chunk partials (fixed order)
 __device__ inline void merge_row(const RowStat* st, int nch, double inv_temp, float& M, double& Z, int& arg)
@@ -279,19 +284,21 @@ __device__ __noinline__ float2 weight_sum8x2(const T* __restrict__ trow, const T
 template <typename T>
 __device__ __noinline__ int find8(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok, int i0,
                                   int level, int mode, const WalkShared& sh, float k2, double run, double target,
-                                  int& last)
+                                  int& last, double& lo, double& hi)
 {
     float tx[kEpt], dx[kEpt];
     load8(trow, i0, V, vec_ok, tx);
     if (level > 0) load8(drow, i0, V, vec_ok, dx);
     int cand = INT_MAX;
     last = -1;
+    lo = hi = 0.0;
 #pragma unroll
     for (int j = 0; j < kEpt; ++j) {
         const float w = weight_at(tx[j], level > 0 ? dx[j] : 0.f, i0 + j, level, mode, sh, k2);
+        const double before = run;
         run += (double)w;
         if (w > 0.f) last = i0 + j;
-        if (cand == INT_MAX && run > target) cand = i0 + j;
+        if (cand == INT_MAX && run > target) { cand = i0 + j; lo = before; hi = run; }
     }
     return cand;
 }
@@ -339,7 +346,7 @@ __device__ double full_pass(const T* __restrict__ trow, const T* __restrict__ dr
 // Inverse CDF in index order over weight_at(., level) using the strip sums of the last full_pass.
 template <typename T>
 __device__ int locate(const T* __restrict__ trow, const T* __restrict__ drow, int V, bool vec_ok, int level, int mode,
-                      WalkShared& sh, float k2, double u)
+                      WalkShared& sh, float k2, double u, bool& borderline)
 {
     const int tid = threadIdx.x, n_strips = (V + kStrip - 1) / kStrip;
     if (tid == 0) {
@@ -358,7 +365,7 @@ __device__ int locate(const T* __restrict__ trow, const T* __restrict__ drow, in
             cum = 0.0;
             for (int s = 0; s < sel; ++s) cum += sh.strip[s];
         }
-        sh.strip_sel = sel; sh.strip_off = cum; sh.target = target;
+        sh.strip_sel = sel; sh.strip_off = cum; sh.target = target; sh.total = tot;
         sh.pick = INT_MAX; sh.pick_last = -1;
     }
     __syncthreads();
@@ -378,11 +385,21 @@ __device__ int locate(const T* __restrict__ trow, const T* __restrict__ drow, in
     for (int wi = 0; wi < (tid >> 5); ++wi) off += sh.scan[wi];
     const double run = off + (incl - loc);
     int last;
-    const int cand = find8(trow, drow, V, vec_ok, i0, level, mode, sh, k2, run, sh.target, last);
+    double lo, hi;
+    const int cand = find8(trow, drow, V, vec_ok, i0, level, mode, sh, k2, run, sh.target, last, lo, hi);
     if (cand != INT_MAX) atomicMin(&sh.pick, cand);
     if (last >= 0) atomicMax(&sh.pick_last, last);
     __syncthreads();
+    if (cand != INT_MAX && cand == sh.pick) { sh.pick_lo = lo; sh.pick_hi = hi; }
+    __syncthreads();
     int res = sh.pick != INT_MAX ? sh.pick : (sh.pick_last >= 0 ? sh.pick_last : 0);
+    // how close the draw came to an edge of the chosen entry's cell of the normalised CDF (a draw
+    // that rounding pushed past the last cell counts as on the edge)
+    if (sh.pick == INT_MAX) borderline = true;
+    else {
+        const double dlo = fabs(u - sh.pick_lo / sh.total), dhi = fabs(sh.pick_hi / sh.total - u);
+        borderline = fmin(dlo, dhi) < kBorderline;
+    }
     __syncthreads();
     return res;
 }
@@ -541,7 +558,7 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
     const double inv_temp = greedy ? 1.0 : 1.0 / (double)temperature;
     const float k2 = (float)inv_temp * kLog2e;
 
-    if (tid == 0) { sh.cur = 0; sh.len = 0; sh.path[0] = 0; sh.tests = 0; sh.rejections = 0; sh.done = 0; }
+    if (tid == 0) { sh.cur = 0; sh.len = 0; sh.path[0] = 0; sh.tests = 0; sh.rejections = 0; sh.done = 0; sh.border_tests = 0; sh.border_draw = 0; }
     __syncthreads();
 
     int lazy_code = 0;                // statistics on demand: a non-finite logit in a row that was needed
@@ -685,6 +702,7 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
                     }
                     const double ratio = (q == 0.0) ? (p > 0.0 ? INFINITY : 0.0) : p / q;
                     ++sh.tests;
+                    if (fabs(ratio - u) < kBorderline) ++sh.border_tests;
                     if (u < ratio) sh.accepted = c;
                     else {
                         ++sh.rejections;
@@ -721,7 +739,9 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
             // ---- final draw at this node ----
             if (sh.done == 2) { final_level = 0; have_strips = false; }
             if (!have_strips) full_pass(trow, drow, V, vec_ok, final_level, mode, sh, k2);
-            const int pick = locate(trow, drow, V, vec_ok, final_level, mode, sh, k2, u0);
+            bool borderline;
+            const int pick = locate(trow, drow, V, vec_ok, final_level, mode, sh, k2, u0, borderline);
+            if (tid == 0) sh.border_draw = borderline ? 1 : 0;
             if (writer && tid == 0) next_token[b] = pick;
             break;
         }
@@ -760,7 +780,7 @@ __global__ void __launch_bounds__(kWalkThreads) accept_walk_kernel(
         }
         if (counters) {
             counters[4 * b] = sh.tests; counters[4 * b + 1] = sh.rejections;
-            counters[4 * b + 2] = 0; counters[4 * b + 3] = 0;
+            counters[4 * b + 2] = sh.border_tests; counters[4 * b + 3] = sh.border_draw;
         }
     }
 }
@@ -841,7 +861,7 @@ __global__ void __launch_bounds__(kWalkThreads) match_walk_kernel(
     const float k2 = (greedy ? 1.f : 1.f / temperature) * kLog2e;
     int32_t* pth = path + (size_t)b * kPathLen;
 
-    if (tid == 0) { sh.code = INT_MAX; sh.cur = 0; sh.len = 0; sh.path[0] = 0; sh.tests = 0; sh.accepted = 0; sh.done = 0; sh.next = -1; }
+    if (tid == 0) { sh.code = INT_MAX; sh.cur = 0; sh.len = 0; sh.path[0] = 0; sh.tests = 0; sh.accepted = 0; sh.done = 0; sh.next = -1; sh.border_tests = 0; }
     __syncthreads();
     if (tid < Tn) {
         const int p = par[tid];
@@ -862,15 +882,17 @@ __global__ void __launch_bounds__(kWalkThreads) match_walk_kernel(
         max_pass(trow, V, vec_ok, sh, M, arg, flag);
         if (flag) { code = CONFU_ST_NONFINITE; break; }
         int x = arg;
+        bool borderline = false;
         if (!greedy) {
             // weights 2^((x - M) k2), unnormalised: the inverse CDF scales the uniform by their sum
             if (tid == 0) { sh.Mt = M; sh.invZt = 1.f; }
             __syncthreads();
             full_pass(trow, trow, V, vec_ok, 0, 0, sh, k2);
-            x = locate(trow, trow, V, vec_ok, 0, 0, sh, k2, (double)uniforms[(size_t)b * Tn + cur]);
+            x = locate(trow, trow, V, vec_ok, 0, 0, sh, k2, (double)uniforms[(size_t)b * Tn + cur], borderline);
         }
         if (tid == 0) {
             ++sh.tests;
+            if (borderline) ++sh.border_tests;
             int hit = -1;
             for (int c = cur + 1; c < Tn; ++c)
                 if (par[c] == cur && tok[c] == x) { hit = c; break; }
@@ -903,7 +925,7 @@ __global__ void __launch_bounds__(kWalkThreads) match_walk_kernel(
                     if (own[k] == a) { fr = Tn + k; break; }
             future_row[b] = fr;
         }
-        if (counters) { counters[4 * b] = sh.tests; counters[4 * b + 1] = sh.accepted; counters[4 * b + 2] = 0; counters[4 * b + 3] = 0; }
+        if (counters) { counters[4 * b] = sh.tests; counters[4 * b + 1] = sh.accepted; counters[4 * b + 2] = sh.border_tests; counters[4 * b + 3] = 0; }
     }
 }
 
@@ -915,12 +937,12 @@ static cudaError_t launch_match_t(int B, int Tn, int C, int V, const void* tl, c
 {
     if (B == 0) return cudaSuccess;
     const size_t smem = sizeof(WalkShared);
-    static bool attr_done[2] = {false, false};
-    const int ti = sizeof(T) == 2 ? 0 : 1;
-    if (!attr_done[ti]) {
-        cudaError_t e = cudaFuncSetAttribute(match_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static OncePerDevice attr_done;          // (one per instantiation of this template)
+    {
+        cudaError_t e = attr_done.run([&] {
+            return cudaFuncSetAttribute(match_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        });
         if (e != cudaSuccess) return e;
-        attr_done[ti] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)B * kWalkCluster);
@@ -951,7 +973,7 @@ cudaError_t launch_accept_match(int B, int T, int C, int V, int logit_dtype, con
 }
 
 template <typename T>
-static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, const void* dl, const int32_t* tokens,
+static cudaError_t launch_accept_t(int sm_count, int B, int Tn, int C, int V, const void* tl, const void* dl, const int32_t* tokens,
                                    const int32_t* parent, const int32_t* con_owner, const float* uniforms,
                                    float temperature, int mode_flags, int32_t* accept_len, int32_t* path,
                                    int32_t* next_token, int32_t* future_row, int32_t* counters, void* workspace,
@@ -963,7 +985,7 @@ static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, 
     const int n_rows = B * Tn;
     const int nmat = greedy ? 1 : 2;
     // enough CTAs to fill the machine a few times over, chunks a multiple of the vector width
-    int nch = (148 * 8 + n_rows * nmat - 1) / (n_rows * nmat);
+    int nch = (sm_count * 8 + n_rows * nmat - 1) / (n_rows * nmat);
     nch = nch < 1 ? 1 : (nch > kStatChunksMax ? kStatChunksMax : nch);
     int chunk_elems = (V + nch - 1) / nch;
     chunk_elems = (chunk_elems + 15) / 16 * 16;
@@ -978,13 +1000,11 @@ static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, 
         if (e != cudaSuccess) return e;
     }
     const size_t smem = sizeof(WalkShared);
-    static bool attr_done[2] = {false, false};
-    const int ti = sizeof(T) == 2 ? 0 : 1;
-    if (!attr_done[ti]) {
-        e = cudaFuncSetAttribute(accept_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_done[ti] = true;
-    }
+    static OncePerDevice attr_done;          // (one per instantiation of this template)
+    e = attr_done.run([&] {
+        return cudaFuncSetAttribute(accept_walk_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    });
+    if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)B * kWalkCluster);
     cfg.blockDim = dim3(kWalkThreads);
@@ -1002,17 +1022,40 @@ static cudaError_t launch_accept_t(int B, int Tn, int C, int V, const void* tl, 
                               counters, status);
 }
 
-cudaError_t launch_accept(const Ctx*, int B, int T, int C, int V, int logit_dtype, const void* tl, const void* dl,
+// SM count of the current device, asked once per device (for callers without a context).
+static cudaError_t current_sm_count(int& n)
+{
+    static int cached[OncePerDevice::kMaxDevices] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= OncePerDevice::kMaxDevices) return cudaErrorInvalidDevice;
+    if (!cached[dev]) {
+        int v = 0;
+        e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        cached[dev] = v;
+    }
+    n = cached[dev];
+    return cudaSuccess;
+}
+
+cudaError_t launch_accept(const Ctx* ctx, int B, int T, int C, int V, int logit_dtype, const void* tl, const void* dl,
                           const int32_t* tokens, const int32_t* parent, const int32_t* con_owner,
                           const float* uniforms, float temperature, int sibling_mode, int32_t* accept_len,
                           int32_t* path, int32_t* next_token, int32_t* future_row, int32_t* counters,
                           void* workspace, int32_t* status, cudaStream_t st)
 {
+    int sm_count = ctx ? ctx->sm_count : 0;
+    if (!ctx) {
+        cudaError_t e = current_sm_count(sm_count);
+        if (e != cudaSuccess) return e;
+    }
     if (logit_dtype == CONFU_F32)
-        return launch_accept_t<float>(B, T, C, V, tl, dl, tokens, parent, con_owner, uniforms, temperature,
+        return launch_accept_t<float>(sm_count, B, T, C, V, tl, dl, tokens, parent, con_owner, uniforms, temperature,
                                       sibling_mode, accept_len, path, next_token, future_row, counters, workspace,
                                       status, st);
-    return launch_accept_t<__nv_bfloat16>(B, T, C, V, tl, dl, tokens, parent, con_owner, uniforms, temperature,
+    return launch_accept_t<__nv_bfloat16>(sm_count, B, T, C, V, tl, dl, tokens, parent, con_owner, uniforms, temperature,
                                           sibling_mode, accept_len, path, next_token, future_row, counters, workspace,
                                           status, st);
 }

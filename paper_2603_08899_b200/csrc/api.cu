@@ -40,12 +40,30 @@ size_t ws_total(const confu_ctx* ctx, const confu_dims* d)
 }  // namespace
 
 namespace confu {
+cudaError_t launch_bounded_wait(unsigned long long limit_ns, int32_t* status, cudaStream_t st);
 bool tc_attention_supported(const confu_dims& d);
 cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
                                 const void* v_cache, int64_t n_slots, const SlotMap& map,
                                 const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
                                 void* partials, void* out, float* lse, int32_t* status, cudaStream_t st);
 }  // namespace confu
+
+namespace {
+
+// Which attention kernel serves these dims under the context's option: a CONFU_ATTENTION_* value
+// (never _AUTO), or a negative error code when a forced path cannot take them.
+int resolve_attention_path(const confu_ctx* ctx, const confu_dims& d)
+{
+    const bool tc = tc_attention_supported(d);
+    switch (ctx->attention_path) {
+        case CONFU_ATTENTION_GENERIC: return CONFU_ATTENTION_GENERIC;
+        case CONFU_ATTENTION_TENSOR: return tc ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ERR_UNSUPPORTED;
+        case CONFU_ATTENTION_TENSOR_PAIR: return CONFU_ERR_UNSUPPORTED;
+        default: return tc ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ATTENTION_GENERIC;
+    }
+}
+
+}  // namespace
 
 extern "C" {
 
@@ -61,6 +79,8 @@ int confu_create(confu_ctx** out, int device)
     c->block_table = nullptr;
     c->max_pages = 0;
     c->last_error = cudaSuccess;
+    c->attention_path = CONFU_ATTENTION_AUTO;
+    c->wait_ns = 2000000000ull;
     cudaError_t e = cudaSetDevice(device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e != cudaSuccess) {
@@ -102,6 +122,30 @@ int confu_set_paging(confu_ctx* ctx, const int32_t* block_table, int32_t max_pag
     return CONFU_OK;
 }
 
+int confu_set_option(confu_ctx* ctx, int32_t option, int64_t value)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    switch (option) {
+        case CONFU_OPT_ATTENTION_PATH:
+            if (value < CONFU_ATTENTION_AUTO || value > CONFU_ATTENTION_TENSOR_PAIR) return CONFU_ERR_ARG;
+            ctx->attention_path = (int)value;
+            return CONFU_OK;
+        case CONFU_OPT_WAIT_LIMIT_NS:
+            if (value < 1000 || value > 10000000000ll) return CONFU_ERR_ARG;
+            ctx->wait_ns = (unsigned long long)value;
+            return CONFU_OK;
+        default: return CONFU_ERR_ARG;
+    }
+}
+
+int confu_selftest_bounded_wait(confu_ctx* ctx, int64_t limit_ns, int32_t* status, void* stream)
+{
+    if (!ctx || !status) return CONFU_ERR_ARG;
+    if (limit_ns < 1000 || limit_ns > 1000000000ll) return CONFU_ERR_ARG;     // the kernel ends within a second
+    cudaError_t e = launch_bounded_wait((unsigned long long)limit_ns, status, (cudaStream_t)stream);
+    return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
+}
+
 const char* confu_status_string(int code)
 {
     switch (code) {
@@ -120,6 +164,8 @@ const char* confu_status_string(int code)
         case CONFU_ST_TIMEOUT: return "bounded device wait expired";
         case CONFU_ST_DEGENERATE: return "residual distribution without mass";
         case CONFU_ST_TOO_DEEP: return "accepted path longer than CONFU_MAX_DEPTH";
+        case CONFU_ST_BAD_PATH: return "accepted path is not an increasing chain of tree nodes from the root";
+        case CONFU_ST_BAD_PLAN: return "plan was built for another attention path";
         default: return "unknown code";
     }
 }
@@ -167,6 +213,8 @@ int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims, const void* q, 
         misaligned(v_soft) || misaligned(plan))
         return CONFU_ERR_ALIGN;
     if (!ctx->workspace || ctx->workspace_bytes < ws_total(ctx, dims)) return CONFU_ERR_WORKSPACE;
+    const int path = resolve_attention_path(ctx, *dims);
+    if (path < 0) return path;
     cudaStream_t st = (cudaStream_t)stream;
     char* ws = (char*)ctx->workspace;
     const void* use_plan = plan;
@@ -177,7 +225,7 @@ int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims, const void* q, 
         use_plan = own_plan;
     }
     cudaError_t e;
-    if (tc_attention_supported(*dims))
+    if (path == CONFU_ATTENTION_TENSOR)
         e = launch_attention_tc(ctx, *dims, q, k_cache, v_cache, n_slots, map, prefix_len, k_soft, v_soft,
                                 use_plan, ws + ws_partial_offset(dims), out, lse, status, st);
     else
@@ -255,7 +303,7 @@ int confu_kv_compact(confu_ctx* ctx, const confu_dims* dims, int32_t n_layers, v
     const SlotMap map = {seq_start, ctx->block_table, ctx->max_pages};
     if (n_layers > 0 && (!k_cache_layers || !v_cache_layers)) return CONFU_ERR_ARG;
     const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : 4);
-    cudaError_t e = launch_compact(ctx, dims->B, n_layers, row_bytes, k_cache_layers, v_cache_layers, map,
+    cudaError_t e = launch_compact(ctx, dims->B, dims->T, n_layers, row_bytes, k_cache_layers, v_cache_layers, map,
                                    prefix_len, accept_len, path, new_prefix_len, status, (cudaStream_t)stream);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
 }
@@ -279,7 +327,8 @@ int confu_kv_append(confu_ctx* ctx, const confu_dims* dims, const void* k_rows, 
 
 int confu_con_embedding(confu_ctx* ctx, int32_t B, int32_t H_in, int32_t H_out, int32_t n_expert, int32_t k_expert,
                         int32_t dtype, const void* hidden, const void* router_w, const void* router_b,
-                        const void* experts, int32_t renormalize, void* out, int32_t* sel, float* gate, void* stream)
+                        const void* experts, int32_t renormalize, void* out, int32_t* sel, float* gate,
+                        int32_t* status, void* stream)
 {
     if (!ctx) return CONFU_ERR_ARG;
     if (B < 0 || H_in <= 0 || H_out <= 0 || n_expert <= 0 || k_expert <= 0 || k_expert > n_expert) return CONFU_ERR_SHAPE;
@@ -289,7 +338,7 @@ int confu_con_embedding(confu_ctx* ctx, int32_t B, int32_t H_in, int32_t H_out, 
     if (!hidden || !router_w || !experts || !out) return CONFU_ERR_ARG;
     if (misaligned(hidden) || misaligned(router_w) || misaligned(experts) || misaligned(out)) return CONFU_ERR_ALIGN;
     cudaError_t e = launch_con_embedding(B, H_in, H_out, n_expert, k_expert, dtype, hidden, router_w, router_b, experts,
-                                         renormalize != 0, out, sel, gate, (cudaStream_t)stream);
+                                         renormalize != 0, out, sel, gate, status, (cudaStream_t)stream);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
 }
 

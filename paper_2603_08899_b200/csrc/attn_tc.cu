@@ -18,25 +18,27 @@
 // does not cover a whole pair writes an unnormalised partial (O, m, l) that combine_kernel merges
 // in a fixed order.
 //
+// The last key tile of a sequence reaches past its last slot, into slots that belong to another
+// sequence, to an unused page tail or to memory nobody ever wrote.  Their scores are masked, so
+// their weights are exactly 0, but 0 x NaN would still poison P V: a spare warp zeroes those rows
+// of the V tile in shared memory before the tensor pipe reads them.  What such slots hold is
+// therefore irrelevant.
+//
 // Every wait on an mbarrier is bounded (wall-clock limit); on expiry the CTA raises an abort flag,
 // every role leaves its loop, tensor memory is released and CONFU_ST_TIMEOUT is reported.
-#include <cuda.h>
-#include <stdlib.h>
-
-#include "attn_tc.cuh"
+#include "tc_ptx.cuh"
 
 namespace confu {
 
 namespace tc {
 
-constexpr int kThreads = 384;            // warps 0-3: softmax of M tile 0, 4-7: of M tile 1, 8: TMA, 9: MMA
+constexpr int kThreads = 384;            // warps 0-3: softmax of M tile 0, 4-7: of M tile 1, 8: TMA, 9: MMA, 10: ragged tail of V
 constexpr int kStages = 2;               // ring of stages; stage g = [V of the CTA's g-1st key tile | K of its g-th]
 constexpr int kTileBytes = kTileKeys * kD * 2;      // 32 KB
 constexpr int kHalfTile = kTileBytes / 2;           // one 64-wide half of the head dim: [128 rows][128 B]
 constexpr int kQBytes = 2 * kTileBytes;             // two M tiles
 constexpr uint32_t kTmemCols = 512;                 // S0 | S1 | O0 | O1, 128 columns each; P_t overlays S_t
 constexpr float kRescaleThreshold = 8.f;            // lazy rescale: move the reference max only past 2^8
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct SharedStorage {
     alignas(1024) uint8_t q[kQBytes];
@@ -44,137 +46,13 @@ struct SharedStorage {
     alignas(8) uint64_t q_full, q_empty;
     uint64_t kv_full[kStages], kv_empty[kStages];
     uint64_t s_full[2], p_full[2], o_done[2];
+    uint64_t v_fixed;                     // the rows of a V tile past the sequence's last slot have been zeroed
     uint32_t tmem_base;
     int abort;
     // per softmax warp: a 32 x 32 fp32 tile for turning "one thread per row" into whole-line stores;
     // the four floats (row, 4q .. 4q+3) sit at float4 index row * 8 + (q ^ (row & 7))
     alignas(16) float4 xpose[8][32 * 8];
 };
-
-// ------------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: false when the wait expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0) {
-            if (*abort) return false;
-            if (global_ns() - t0 > kWaitLimitNs) { *abort = 1; return false; }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
-        : "memory");
-}
-
-// high word of every shared-memory descriptor: SBO = 1024 B (>> 4) | version 1 (bit 46) | swizzle 128B (code 2, bits 61-63)
-constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint64_t* bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
-}
-// Shared-memory matrix descriptors are passed as their two 32-bit words: the low word carries the
-// start address and the leading byte offset (both >> 4), the high word is the same for every
-// operand of this kernel (stride byte offset 1024, descriptor version 1, 128-byte swizzle).
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(acc), "r"(kDescHi)
-        : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t acc)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-        "mov.b64 db, {%2, %5};\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(acc), "r"(kDescHi)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
-        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
-          "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-          "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
-        : "memory");
-}
-
-// Low word of a shared-memory matrix descriptor: start address and leading byte offset, both >> 4.
-// K-major operands (Q, K) ignore the leading offset (16 B by convention); the MN-major V tile uses
-// it as the distance between its two 64-column halves.
-__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo) { return ((addr >> 4) & 0x3FFFu) | ((lbo >> 4) << 16); }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; B K-major (QK^T) or MN-major (PV).
-constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
 
 // ------------------------------------------------------------------------------------ work list
 struct Segment {
@@ -217,6 +95,14 @@ struct Walker {
     }
 };
 
+// Slots of key tile `tile` that belong to the sequence when the tile is its last key tile and
+// reaches past its last slot (1..127); 0 for every other tile.
+__device__ __forceinline__ int ragged_rows(const Segment& s, int tile, int R)
+{
+    if (tile != s.nkt - 1) return 0;
+    return (int)((s.P + R) & (kTileKeys - 1));
+}
+
 // ------------------------------------------------------------------------------------ roles
 // Key tiles of the CTA's share, all pairs together, are numbered g = 0..n-1 in walking order; stage
 // g of the ring carries V of tile g-1 and K of tile g (stage 0 has no V, stage n no K).
@@ -240,7 +126,7 @@ __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanVi
     // fills stage `stage` with V of `prev` (if any) and K of `cur` (if any)
     auto fill = [&](const TileRef* cur) -> bool {
         const uint32_t st = stage % kStages;
-        if (!mbar_wait(&sh.kv_empty[st], ((stage / kStages) & 1) ^ 1, &sh.abort)) return false;
+        if (!mbar_wait(&sh.kv_empty[st], ((stage / kStages) & 1) ^ 1, &sh.abort, prm.wait_ns)) return false;
         mbar_arrive_expect_tx(&sh.kv_full[st], (have_prev ? kTileBytes : 0) + (cur ? kTileBytes : 0));
         if (have_prev) {
             const CUtensorMap* m = prev.soft ? vs_map : v_map;
@@ -268,7 +154,7 @@ __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanVi
             // the Q buffer), then, at the start of a pair, its Q (both M tiles, two 64-wide halves each)
             if (!fill(&cur)) return;
             if (t == s.t0) {
-                if (!mbar_wait(&sh.q_empty, (seg & 1) ^ 1, &sh.abort)) return;
+                if (!mbar_wait(&sh.q_empty, (seg & 1) ^ 1, &sh.abort, prm.wait_ns)) return;
                 mbar_arrive_expect_tx(&sh.q_full, 2u * prm.n_mt * q_box_bytes);
                 for (int mt = 0; mt < prm.n_mt; ++mt)
                     for (int kb = 0; kb < 2; ++kb)
@@ -315,11 +201,17 @@ __device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& p
                    (first_of_segment && i == 0) ? 0u : 1u);
     };
     // one stage: P V of the previous key tile (if any), Q K^T of the current one (if any)
-    bool have_prev = false, prev_first = false, prev_last = false;
-    auto run_stage = [&](bool have_cur, bool cur_first, bool cur_last) -> bool {
+    bool have_prev = false, prev_first = false, prev_last = false, prev_ragged = false;
+    uint32_t n_fix = 0;
+    auto run_stage = [&](bool have_cur, bool cur_first, bool cur_last, bool cur_ragged) -> bool {
         const uint32_t st = stage % kStages;
-        if (!mbar_wait(&sh.kv_full[st], (stage / kStages) & 1, &sh.abort)) return false;
-        if (have_cur && cur_first && !mbar_wait(&sh.q_full, seg & 1, &sh.abort)) return false;
+        if (!mbar_wait(&sh.kv_full[st], (stage / kStages) & 1, &sh.abort, prm.wait_ns)) return false;
+        if (have_cur && cur_first && !mbar_wait(&sh.q_full, seg & 1, &sh.abort, prm.wait_ns)) return false;
+        // the V tile of a sequence's last key tile: wait until its rows past the last slot are zero
+        if (have_prev && prev_ragged) {
+            if (!mbar_wait(&sh.v_fixed, n_fix & 1, &sh.abort, prm.wait_ns)) return false;
+            ++n_fix;
+        }
         tc_fence_after();
         const uint32_t vl = v_lo0 + st * kStageStep, kl = k_lo0 + st * kStageStep;
 #pragma unroll
@@ -327,7 +219,7 @@ __device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& p
             if (have_prev) {
                 // (At the start of a pair this P V overwrites the previous pair's O_t; the softmax
                 // threads hand P over only after they have read that O_t out.)
-                if (!mbar_wait(&sh.p_full[t], (stage - 1) & 1, &sh.abort)) return false;
+                if (!mbar_wait(&sh.p_full[t], (stage - 1) & 1, &sh.abort, prm.wait_ns)) return false;
                 tc_fence_after();
                 issue_pv(t, vl, prev_first);
                 if (prev_last) tc_commit(&sh.o_done[t]);
@@ -340,16 +232,55 @@ __device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& p
         have_prev = have_cur;
         prev_first = cur_first;
         prev_last = cur_last;
+        prev_ragged = cur_ragged;
         return true;
     };
 
+    const int R = prm.d.T + prm.d.C;
     while (w.next(s)) {
         const int n_tiles = s.t1 - s.t0;
         for (int j = 0; j < n_tiles; ++j)
-            if (!run_stage(true, j == 0, j + 1 == n_tiles)) return;
+            if (!run_stage(true, j == 0, j + 1 == n_tiles, ragged_rows(s, s.t0 + j, R) > 0)) return;
         ++seg;
     }
-    if (have_prev) run_stage(false, false, false);
+    if (have_prev) run_stage(false, false, false, false);
+}
+
+// Follows the stages of the ring like the issuing thread does and, where a stage carries the V tile
+// of a sequence's last key tile, zeroes the rows past the sequence's last slot (generic-proxy
+// stores, made visible to the tensor pipe by a proxy fence) before it lets the issuing thread go on.
+// It arrives on every stage's empty barrier, so a stage is never refilled before it has seen it.
+__device__ void tail_role(SharedStorage& sh, const Params& prm, const PlanView& pv)
+{
+    Walker w(pv, prm, blockIdx.x);
+    Segment s;
+    const int R = prm.d.T + prm.d.C, lane = threadIdx.x & 31;
+    uint32_t stage = 0;
+    int prev_valid = 0;                 // > 0: the previous tile's V needs rows [prev_valid, 128) zeroed
+    bool have_prev = false;
+    auto run_stage = [&](int cur_valid) -> bool {
+        const uint32_t st = stage % kStages;
+        if (!mbar_wait(&sh.kv_full[st], (stage / kStages) & 1, &sh.abort, prm.wait_ns)) return false;
+        if (have_prev && prev_valid > 0) {
+            const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+            for (int half = 0; half < 2; ++half)
+                for (int off = prev_valid * 128 + lane * 16; off < kHalfTile; off += 32 * 16)
+                    *reinterpret_cast<uint4*>(sh.kv[st][0] + half * kHalfTile + off) = zero;
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.v_fixed);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.kv_empty[st]);
+        ++stage;
+        have_prev = true;
+        prev_valid = cur_valid;
+        return true;
+    };
+    while (w.next(s))
+        for (int tile = s.t0; tile < s.t1; ++tile)
+            if (!run_stage(ragged_rows(s, tile, R))) return;
+    if (have_prev) run_stage(0);
 }
 
 // Which of the 128 keys of tile `t` may row r see.  lo: keys 0..63 of the tile, hi: 64..127.
@@ -433,7 +364,7 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
         const uint64_t mask = row_valid ? pv.mask[(size_t)s.b * kMaxRows + r] : 0ull;
         float m_ref = -INFINITY, l = 0.f;
         for (int tile = s.t0; tile < s.t1; ++tile) {
-            if (!mbar_wait(&sh.s_full[t], n_s & 1, &sh.abort)) return;
+            if (!mbar_wait(&sh.s_full[t], n_s & 1, &sh.abort, prm.wait_ns)) return;
             ++n_s;
             tc_fence_after();
             uint32_t sv[128];
@@ -484,7 +415,7 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
             mbar_arrive(&sh.p_full[t]);
         }
         // ---- epilogue of this pair / range ----
-        if (!mbar_wait(&sh.o_done[t], seg & 1, &sh.abort)) return;
+        if (!mbar_wait(&sh.o_done[t], seg & 1, &sh.abort, prm.wait_ns)) return;
         tc_fence_after();
         // O_t leaves tensor memory one row per thread; written like that, every store instruction of a
         // warp would touch 32 different lines.  Each 32-column chunk goes through the warp's
@@ -570,7 +501,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     if (threadIdx.x == 0) {
         mbar_init(&sh.q_full, 1);
         mbar_init(&sh.q_empty, 1);
-        for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 1); }
+        // a stage is free again when its MMAs have completed and the tail warp has seen it
+        for (int i = 0; i < kStages; ++i) { mbar_init(&sh.kv_full[i], 1); mbar_init(&sh.kv_empty[i], 2); }
+        mbar_init(&sh.v_fixed, 1);
         for (int t = 0; t < 2; ++t) {
             mbar_init(&sh.s_full[t], 1);
             mbar_init(&sh.p_full[t], 128);
@@ -604,6 +537,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
                 if (prm.n_mt > 1) mma_role<true>(sh, prm, pv, tmem);
                 else mma_role<false>(sh, prm, pv, tmem);
             }
+        } else if (warp == 10) {
+            tail_role(sh, prm, pv);
         }
         __syncwarp();
     }
@@ -661,8 +596,6 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
 
 bool tc_attention_supported(const confu_dims& d)
 {
-    static const bool force_generic = getenv("CONFU_FORCE_GENERIC") != nullptr;     // debugging aid
-    if (force_generic) return false;
     const int G = d.Hq / d.Hkv;
     return d.kv_dtype == CONFU_BF16 && d.D == 128 && G <= 4 && d.S <= 128;
 }
@@ -693,12 +626,14 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     prm.n_rg = (R + kGroupRows - 1) / kGroupRows;
     prm.G = G;
     prm.c = (d.sm_scale != 0.f ? d.sm_scale : 1.f / sqrtf((float)d.D)) * 1.4426950408889634f;
+    prm.wait_ns = ctx->wait_ns;
     const size_t smem = sizeof(SharedStorage) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static OncePerDevice attr_done;
+    {
+        cudaError_t e = attr_done.run([&] {
+            return cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        });
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     // Launched as a programmatic dependent of whatever precedes it in the stream: its CTAs may be
     // scheduled while the predecessor drains; the kernel waits (griddepcontrol.wait, first thing) for

@@ -22,6 +22,7 @@ struct Params {
     int n_rg;            // groups of 64 query rows (R > 64 ? 2 : 1); a pair = (sequence, kv head, row group)
     int G;
     float c;             // sm_scale * log2(e)
+    unsigned long long wait_ns;   // limit of every wait on an mbarrier (wall clock)
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)

@@ -6,6 +6,17 @@
 namespace confu {
 namespace tc {
 
+// Output row (b, r, head g * G + hl) and its lse as zeros, by one warp: what a sequence with a
+// malformed tree gets (the same as on the generic path).
+__device__ __forceinline__ void zero_row(const Params& prm, int b, int g, int r, int hl, int lane)
+{
+    const int R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
+    if (r >= R) return;
+    const int h = g * prm.G + hl;
+    reinterpret_cast<uint2*>(prm.out + (((size_t)b * R + r) * Hq + h) * kD)[lane] = make_uint2(0u, 0u);
+    if (prm.lse && lane == 0) prm.lse[((size_t)b * R + r) * Hq + h] = 0.f;
+}
+
 // Merge of the split-KV partials of one (sequence, kv head) pair, in CTA order (deterministic).
 // One block per (pair, M tile, 32 rows); a warp takes a row at a time (four rows in all), lane i the
 // row's columns 4i..4i+3, so partial rows are read and output rows written as whole 512- and
@@ -19,14 +30,19 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
     const int per_seq = prm.d.Hkv * prm.n_rg;
     const int b = pair / per_seq, g = (pair % per_seq) / prm.n_rg, rg = pair % prm.n_rg;
     const int nt = pv.tiles[b];
-    if (nt == 0 || t >= prm.n_mt) return;
+    if (t >= prm.n_mt) return;
+    const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (nt == 0) {                                      // malformed tree: no CTA worked on the pair; its rows read 0
+        for (int lane_row = blockIdx.z * 32 + warp; lane_row < min(32 * G, (int)blockIdx.z * 32 + 32); lane_row += 8)
+            zero_row(prm, b, g, kGroupRows * rg + 32 * t + lane_row / G, lane_row % G, lane);
+        return;
+    }
     const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
     // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
     const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
     const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
     if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
-    const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const size_t slot_floats = partial_slot_bytes() / sizeof(float);
     for (int lane_row = blockIdx.z * 32 + warp; lane_row < min(32 * G, (int)blockIdx.z * 32 + 32); lane_row += 8) {
         const int r = kGroupRows * rg + 32 * t + lane_row / G, hl = lane_row % G;
@@ -72,17 +88,21 @@ __global__ void __launch_bounds__(32 * kCombineRowsPerBlock) combine_wide_kernel
     const int per_seq = prm.d.Hkv * prm.n_rg;
     const int b = pair / per_seq, g = (pair % per_seq) / prm.n_rg, rg = pair % prm.n_rg;
     const int nt = pv.tiles[b];
-    if (nt == 0 || t >= prm.n_mt) return;
-    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
-    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
-    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
-    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
-    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
+    if (t >= prm.n_mt) return;
     const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int lane_row = blockIdx.z * kCombineRowsPerBlock + warp;
     const int r = kGroupRows * rg + 32 * t + lane_row / G, hl = lane_row % G;
     if (lane_row >= 32 * G || r >= R) return;
+    if (nt == 0) {                                      // malformed tree: no CTA worked on the pair; its rows read 0
+        zero_row(prm, b, g, r, hl, lane);
+        return;
+    }
+    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
+    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
+    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
+    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
+    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
     const int row = t * 128 + lane_row;
     const int n_parts = c_last - c_first + 1;
     const size_t slot_floats = partial_slot_bytes() / sizeof(float);

@@ -121,6 +121,26 @@ struct Ctx {
     const int32_t* block_table;    // paged pools when set (confu_set_paging)
     int32_t max_pages;
     cudaError_t last_error;
+    int attention_path;            // CONFU_ATTENTION_* (confu_set_option)
+    unsigned long long wait_ns;    // limit of the bounded waits inside the kernels
+};
+
+// A function attribute (the opt-in to more than 48 KB of dynamic shared memory) belongs to a
+// device, not to the process: run `fn` once for every device that comes along as the current one.
+struct OncePerDevice {
+    static constexpr int kMaxDevices = 64;
+    bool done[kMaxDevices] = {};
+    template <typename F> cudaError_t run(F fn)
+    {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        if (done[dev]) return cudaSuccess;
+        e = fn();
+        if (e == cudaSuccess) done[dev] = true;
+        return e;
+    }
 };
 
 // ---------------------------------------------------------------------------
@@ -207,14 +227,14 @@ cudaError_t launch_accept_match(int B, int T, int C, int V, int logit_dtype, con
                                 float temperature, int32_t* accept_len, int32_t* path, int32_t* next_token,
                                 int32_t* future_row, int32_t* counters, int32_t* status, cudaStream_t st);
 
-cudaError_t launch_compact(const Ctx* ctx, int B, int n_layers, int64_t row_bytes, void* const* k_layers,
+cudaError_t launch_compact(const Ctx* ctx, int B, int T, int n_layers, int64_t row_bytes, void* const* k_layers,
                            void* const* v_layers, const SlotMap& map, const int32_t* prefix_len,
                            const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len,
                            int32_t* status, cudaStream_t st);
 
 cudaError_t launch_con_embedding(int B, int H_in, int H_out, int n_expert, int k_expert, int dtype, const void* hidden,
                                  const void* router_w, const void* router_b, const void* experts, int renormalize,
-                                 void* out, int32_t* sel, float* gate, cudaStream_t st);
+                                 void* out, int32_t* sel, float* gate, int32_t* status, cudaStream_t st);
 
 cudaError_t launch_append(int B, int R, int64_t row_bytes, const void* k_rows, const void* v_rows, void* k_cache,
                           void* v_cache, const SlotMap& map, const int32_t* prefix_len, cudaStream_t st);

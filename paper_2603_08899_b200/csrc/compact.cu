@@ -7,30 +7,48 @@
 // 16-byte column of the row and walks k upwards in batches (all loads of a batch before its
 // stores), so within a thread every source is read before any step at or after it overwrites
 // that slot, and different threads never touch each other's columns.
+//
+// That argument needs path[0] = 0 < path[1] < ... < path[a] < T and a <= CONFU_MAX_DEPTH.  A path
+// that breaks it (a stale or corrupted buffer) is not followed: the sequence gets the status code
+// CONFU_ST_BAD_PATH, nothing of it is copied and its new prefix length is prefix_len + 1 (the root
+// only).  Every thread checks the path itself (at most 64 cached loads), so no thread copies a row
+// of a path another thread would have refused.
 #include "common.cuh"
 
 namespace confu {
 
 constexpr int kCompactBatch = 8;
 
-__global__ void __launch_bounds__(128) compact_kernel(int n_layers, int64_t row_vecs, void* const* __restrict__ k_layers,
+__global__ void __launch_bounds__(128) compact_kernel(int n_layers, int T, int64_t row_vecs, void* const* __restrict__ k_layers,
                                                       void* const* __restrict__ v_layers,
                                                       const SlotMap map,
                                                       const int32_t* __restrict__ prefix_len,
                                                       const int32_t* __restrict__ accept_len,
                                                       const int32_t* __restrict__ path,
-                                                      int32_t* __restrict__ new_prefix_len)
+                                                      int32_t* __restrict__ new_prefix_len,
+                                                      int32_t* __restrict__ status)
 {
     const int b = blockIdx.z, layer = blockIdx.y >> 1, kv = blockIdx.y & 1;
     const int64_t col = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int32_t* pth = path + (size_t)b * kPathLen;
     int a = accept_len[b];
-    a = a < 0 ? 0 : (a > CONFU_MAX_DEPTH ? CONFU_MAX_DEPTH : a);
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0 && new_prefix_len)
-        new_prefix_len[b] = prefix_len[b] + a + 1;
+    bool ok = a >= 0 && a <= CONFU_MAX_DEPTH && pth[0] == 0;
+    if (ok) {
+        int before = 0;
+        for (int k = 1; k <= a; ++k) {
+            const int node = pth[k];
+            ok = ok && node > before && node < T;
+            before = node;
+        }
+    }
+    if (!ok) a = 0;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        if (new_prefix_len) new_prefix_len[b] = prefix_len[b] + a + 1;
+        if (!ok && status) status[b] = CONFU_ST_BAD_PATH;
+    }
     if (a == 0 || col >= row_vecs) return;
     uint4* pool = reinterpret_cast<uint4*>(kv ? v_layers[layer] : k_layers[layer]);
     const int64_t root = prefix_len[b];              // the root's slot, counted from the sequence's first
-    const int32_t* pth = path + (size_t)b * kPathLen;
     for (int k0 = 1; k0 <= a; k0 += kCompactBatch) {
         uint4 buf[kCompactBatch];
 #pragma unroll
@@ -64,21 +82,21 @@ cudaError_t launch_append(int B, int R, int64_t row_bytes, const void* k_rows, c
     return cudaGetLastError();
 }
 
-cudaError_t launch_compact(const Ctx*, int B, int n_layers, int64_t row_bytes, void* const* k_layers,
+cudaError_t launch_compact(const Ctx*, int B, int T, int n_layers, int64_t row_bytes, void* const* k_layers,
                            void* const* v_layers, const SlotMap& map, const int32_t* prefix_len,
                            const int32_t* accept_len, const int32_t* path, int32_t* new_prefix_len,
-                           int32_t* /*status*/, cudaStream_t st)
+                           int32_t* status, cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
     const int64_t row_vecs = row_bytes / 16;
     // with no layers there is still new_prefix_len to write: one block row does it
     dim3 grid((unsigned)((row_vecs + 127) / 128), (unsigned)(n_layers > 0 ? 2 * n_layers : 1), (unsigned)B);
     if (n_layers == 0) {
-        compact_kernel<<<dim3(1, 1, B), 128, 0, st>>>(0, 0, k_layers, v_layers, map, prefix_len, accept_len, path,
-                                                       new_prefix_len);
+        compact_kernel<<<dim3(1, 1, B), 128, 0, st>>>(0, T, 0, k_layers, v_layers, map, prefix_len, accept_len, path,
+                                                       new_prefix_len, status);
     } else {
-        compact_kernel<<<grid, 128, 0, st>>>(n_layers, row_vecs, k_layers, v_layers, map, prefix_len, accept_len,
-                                             path, new_prefix_len);
+        compact_kernel<<<grid, 128, 0, st>>>(n_layers, T, row_vecs, k_layers, v_layers, map, prefix_len, accept_len,
+                                             path, new_prefix_len, status);
     }
     return cudaGetLastError();
 }

@@ -7,6 +7,12 @@
 // the same for every sequence and stays in L2.  The softmax and the selection (k rounds of a warp
 // argmax, the lower index on equal scores) run in one warp; the output is written 16 bytes per
 // thread.  A few hundred KB per sequence: the kernel is bound by latency, not by bandwidth.
+//
+// A non-finite router score (a NaN or an infinity in the hidden state or the router) makes the
+// scores of the sequence meaningless: the sequence's output row is written as zeros, its selection
+// as experts 0..k-1 with gate 0, and status[b] (optional) gets CONFU_ST_NONFINITE.  The selected
+// indices are clamped to the table whatever the scores are, so no input value can send a load or a
+// store out of bounds.
 #include "common.cuh"
 
 namespace confu {
@@ -40,16 +46,19 @@ template <typename T>
 __global__ void __launch_bounds__(kMoeThreads) con_embedding_kernel(
     int H_in, int H_out, int n_expert, int k_expert, const T* __restrict__ hidden, const T* __restrict__ router_w,
     const T* __restrict__ router_b, const T* __restrict__ experts, int renormalize, T* __restrict__ out,
-    int32_t* __restrict__ sel, float* __restrict__ gate)
+    int32_t* __restrict__ sel, float* __restrict__ gate, int32_t* __restrict__ status)
 {
     constexpr int kVec = Vec16<T>::n;
     __shared__ float s_score[kMoeMaxExperts];
     __shared__ int s_sel[kMoeMaxK];
     __shared__ float s_w[kMoeMaxK];
+    __shared__ int s_bad;
     const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const T* h = hidden + (size_t)b * H_in;
     const bool vec_in = H_in % kVec == 0, vec_out = H_out % kVec == 0;
 
+    if (tid == 0) s_bad = 0;
+    __syncthreads();
     // ---- router logits ----
     for (int e = warp; e < n_expert; e += kMoeThreads / 32) {
         const T* w = router_w + (size_t)e * H_in;
@@ -66,9 +75,23 @@ __global__ void __launch_bounds__(kMoeThreads) con_embedding_kernel(
             for (int i = lane; i < H_in; i += 32) acc = fmaf(to_f32(h[i]), to_f32(w[i]), acc);
         }
         acc = warp_sum(acc);
-        if (lane == 0) s_score[e] = acc + (router_b ? to_f32(router_b[e]) : 0.f);
+        if (lane == 0) {
+            const float sc = acc + (router_b ? to_f32(router_b[e]) : 0.f);
+            s_score[e] = sc;
+            if (!(fabsf(sc) <= 3.0e38f)) s_bad = 1;
+        }
     }
     __syncthreads();
+    if (s_bad) {
+        T* o = out + (size_t)b * H_out;
+        for (int j = tid; j < H_out; j += kMoeThreads) o[j] = from_f32<T>(0.f);
+        if (tid < k_expert) {
+            if (sel) sel[(size_t)b * k_expert + tid] = tid;
+            if (gate) gate[(size_t)b * k_expert + tid] = 0.f;
+        }
+        if (tid == 0 && status) status[b] = CONFU_ST_NONFINITE;
+        return;
+    }
 
     // ---- softmax and the k largest scores (one warp) ----
     if (warp == 0) {
@@ -98,6 +121,7 @@ __global__ void __launch_bounds__(kMoeThreads) con_embedding_kernel(
                 const int oe = __shfl_xor_sync(0xffffffffu, be, o);
                 if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
             }
+            be = min(max(be, 0), n_expert - 1);       // finite scores always give an index; never trust that for an address
             if (lane == 0) {
                 s_sel[k] = be;
                 s_w[k] = bv * inv_z;
@@ -143,17 +167,17 @@ __global__ void __launch_bounds__(kMoeThreads) con_embedding_kernel(
 
 cudaError_t launch_con_embedding(int B, int H_in, int H_out, int n_expert, int k_expert, int dtype, const void* hidden,
                                  const void* router_w, const void* router_b, const void* experts, int renormalize,
-                                 void* out, int32_t* sel, float* gate, cudaStream_t st)
+                                 void* out, int32_t* sel, float* gate, int32_t* status, cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
     if (dtype == CONFU_F32)
         con_embedding_kernel<float><<<B, kMoeThreads, 0, st>>>(H_in, H_out, n_expert, k_expert, (const float*)hidden,
                                                                (const float*)router_w, (const float*)router_b,
-                                                               (const float*)experts, renormalize, (float*)out, sel, gate);
+                                                               (const float*)experts, renormalize, (float*)out, sel, gate, status);
     else
         con_embedding_kernel<__nv_bfloat16><<<B, kMoeThreads, 0, st>>>(
             H_in, H_out, n_expert, k_expert, (const __nv_bfloat16*)hidden, (const __nv_bfloat16*)router_w,
-            (const __nv_bfloat16*)router_b, (const __nv_bfloat16*)experts, renormalize, (__nv_bfloat16*)out, sel, gate);
+            (const __nv_bfloat16*)router_b, (const __nv_bfloat16*)experts, renormalize, (__nv_bfloat16*)out, sel, gate, status);
     return cudaGetLastError();
 }
 

@@ -116,9 +116,7 @@ class VerifyStep:
 
 def uses_tensor_core_path(cfg):
     """Mirror of the library's dispatch rule: bf16, head dim 128, at most 4 query heads per KV head."""
-    import os
-    return (cfg.kv_dtype == torch.bfloat16 and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
-            and "CONFU_FORCE_GENERIC" not in os.environ)
+    return cfg.kv_dtype == torch.bfloat16 and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
 
 
 def attention_kernels_per_layer(cfg):

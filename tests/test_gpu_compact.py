@@ -40,7 +40,7 @@ def _run(gpu, dtype, Hkv, D, L, paths, plen_list, R=64, seed=0):
     kp = torch.tensor([t.data_ptr() for t in kd], dtype=torch.int64, device="cuda")
     vp = torch.tensor([t.data_ptr() for t in vd], dtype=torch.int64, device="cuda")
     new_len = torch.zeros(B, dtype=torch.int32, device="cuda")
-    dims = cb.make_dims(B, Hkv, Hkv, D, R - 4, 4, 0, dtype)
+    dims = cb.make_dims(B, Hkv, Hkv, D, R, 0, 0, dtype)          # T = 64: node ids up to 63 are valid
     cb.confu_kv_compact(gpu.ctx, dims, L, kp, vp, seq_start.cuda(), plen.cuda(), alen.cuda(), path.cuda(), new_len,
                         None)
     torch.cuda.synchronize()

@@ -14,6 +14,7 @@ import ctypes as C
 import pytest
 import torch
 
+from oracle import ref
 from paper_2603_08899_b200 import binding as cb
 from paper_2603_08899_b200 import inputs
 from tests import harness as H
@@ -64,6 +65,11 @@ def test_static_scratch_entry_point_matches_the_ordinary_one_on_two_calls_in_a_r
             assert want["status"].tolist() == [0] * cfg.B
             for k in want:
                 assert torch.equal(got[k], want[k]), (cfg.seed, k, got[k], want[k])
+            # and directly against the CPU oracle, under the same rule as every other acceptance test
+            oracle = ref.tree_accept(tl, dl if temperature > 0 else None, tok, parent, owner,
+                                     u if temperature > 0 else None, temperature=temperature, sibling_mode=1)
+            exact, border = H.compare_accept(got, oracle)
+            assert exact + border == cfg.B and border <= 1
     finally:
         gpu.close()
 
