@@ -53,6 +53,33 @@ def step_bytes(cfg, plen, accept_len_mean):
     return cfg.L * attention_bytes_per_layer(cfg, plen) + logits + compact
 
 
+def key_tiles_per_layer(cfg, plen):
+    """128-key tiles one attention launch walks on the tensor-core path: per (sequence, KV head, group of
+    64 query rows) the key tiles of prefix + R slots, plus one tile for the soft prompts."""
+    n_rg = (cfg.R + 63) // 64
+    per_seq = sum((int(p) + cfg.R + 127) // 128 + (1 if cfg.S else 0) for p in plen)
+    return per_seq * cfg.Hkv * n_rg
+
+
+def attention_lens(cfg, plen, launch_s, clocks, peaks, sm_count):
+    """One attention launch against both ceilings.  `bound` is the ceiling that binds at the measured
+    peaks (the larger of bytes / copy bandwidth and FLOPs / sustained bf16 matmul rate)."""
+    a_bytes = attention_bytes_per_layer(cfg, plen)
+    a_flops = attention_flops_per_layer(cfg, plen)
+    t_hbm, t_tc = a_bytes / (peaks["hbm_gbs"] * 1e9), a_flops / (peaks["bf16_tflops"] * 1e12)
+    gbs, tf = a_bytes / launch_s / 1e9, a_flops / launch_s / 1e12
+    mhz = clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None
+    tiles = key_tiles_per_layer(cfg, plen)
+    return {"bound": "tensor" if t_tc > t_hbm else "hbm", "launch_us": launch_s * 1e6,
+            "floor_us": {"hbm": t_hbm * 1e6, "tensor": t_tc * 1e6},
+            "bytes_per_launch": a_bytes, "flops_per_launch": a_flops, "key_tiles_per_launch": tiles,
+            "hbm_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
+            "tensor_tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops"],
+            # clock-independent figures: time x median SM clock under load
+            "mcycles_per_launch": None if mhz is None else launch_s * mhz,
+            "cycles_per_key_tile_per_sm": None if mhz is None else launch_s * mhz * 1e6 * sm_count / max(tiles, 1)}
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -211,7 +238,7 @@ def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sp = oracle_prepare(cfg, target_visits=25e6, max_seqs=4)
+    sp = oracle_prepare(cfg, target_visits=args.reference_visits, max_seqs=args.reference_seqs)
     for i in range(args.warmup):
         oracle_sample(sp)
     t0 = time.perf_counter()
@@ -222,7 +249,10 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "note": "oracle timed on a bounded sample, scaled to a whole step",
+            "config": {"workload": cfg.name, "B": cfg.B, "layers": cfg.L, "heads": f"{cfg.Hq}q/{cfg.Hkv}kv", "head_dim": cfg.D,
+                       "tree_rows": cfg.T, "contemplate_rows": cfg.C, "soft_prompt": cfg.S, "vocab": cfg.V,
+                       "prefix": "ragged U[512,16384]" if isinstance(cfg.prefix, tuple) else cfg.prefix,
+                       "temperature": 1.0, "note": "oracle timed on a bounded sample, scaled to a whole step",
                        "sample_wall_seconds": wall},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": res[0]["cores"], "kind": "oracle",
                              "sample": res[0]["sample"]},
@@ -232,7 +262,7 @@ def run_reference(args, cfg):
 
 
 # ----------------------------------------------------------------------------- GPU leg
-def build_workload(cfg, device, rank):
+def build_workload(cfg, device, rank, temperature=1.0):
     from paper_2603_08899_b200.step import VerifyStep
     cfg = rank_config(cfg, rank)
     parent, owner = inputs.trees(cfg)
@@ -244,7 +274,7 @@ def build_workload(cfg, device, rank):
         q.append(t["q"]); k.append(t["k_cache"]); v.append(t["v_cache"]); ks.append(t["k_soft"]); vs.append(t["v_soft"])
         out.append(torch.empty_like(t["q"]))
     tl, dl = inputs.logits(cfg, device=device)
-    tok = inputs.draft_tokens(cfg, parent, dl, 1.0)
+    tok = inputs.draft_tokens(cfg, parent, dl, temperature)
     u = inputs.uniforms(cfg)
     step = VerifyStep(cfg, n_slots, device=device)
     step.bind(q, k, v, ks if cfg.S else None, vs if cfg.S else None, out, seq_start.to(device), plen.to(device),
@@ -265,6 +295,73 @@ def spot_check(cfg, step, host):
             step.next_token[b].item() == o["next_token"][b].item()
         ok &= bool(same or o["ratio_margin"][b].item() < 1e-5 or o["resample_margin"][b].item() < 1e-5)
     return ok
+
+
+def time_other_workload(name, temperature, device, gpu_index, peaks, min_seconds=1.0):
+    """One more workload of the table, timed as replays of its captured graphs for at least min_seconds
+    (so that the clock sampler sees the load), its KV freed afterwards.  Returns the record that goes
+    under config.workloads[name]."""
+    from paper_2603_08899_b200 import step as step_mod
+    cfg, step, host = build_workload(inputs.CONFIGS[name], device, 0, temperature)
+    plen = host["plen"]
+    for _ in range(3):
+        step.status.zero_()
+        step.run(temperature)
+    torch.cuda.synchronize()
+    status_ok = bool((step.status == 0).all().item())
+    step.capture(temperature)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        step.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    n = int(min(20000, max(20, min_seconds * 1e3 / max(e0.elapsed_time(e1) / 5, 1e-3))))
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n)]
+    sampler = ClockSampler(gpu_index)
+    torch.cuda.synchronize()
+    for i in range(n):
+        step.replay(ev[i])
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = [ev[i][0].elapsed_time(ev[i][4]) for i in range(n)]
+    total_ms = ev[0][0].elapsed_time(ev[n - 1][4])
+    ms_attn = statistics.mean(ev[i][1].elapsed_time(ev[i][2]) for i in range(n))
+    ms_acc = statistics.mean(ev[i][2].elapsed_time(ev[i][3]) for i in range(n))
+    alen = step.accept_len.float().mean().item()
+    sbytes = step_bytes(cfg, plen, alen) if temperature > 0 else \
+        step_bytes(cfg, plen, alen) - cfg.B * cfg.T * cfg.V * step.tl.element_size()       # greedy reads the target matrix only
+    rec = {"temperature": temperature, "steps": n, "ms_per_step": total_ms / n, "ms_per_step_median": statistics.median(ms),
+           "ms_per_step_min": min(ms), "steps_per_sec": n / (total_ms * 1e-3),
+           "parts_ms": {"attention": ms_attn, "accept": ms_acc},
+           "attention": attention_lens(cfg, plen, ms_attn * 1e-3 / cfg.L, clocks, peaks, step_mod.sm_count(step)),
+           "step_bytes": sbytes, "step_frac_of_measured_hbm": sbytes / (total_ms / n * 1e-3) / 1e9 / peaks["hbm_gbs"],
+           "mcycles_per_step": None if not clocks.get("sm_mhz") else total_ms / n * 1e-3 * clocks["sm_mhz"],
+           "mean_accept_len": alen, "status_ok": status_ok, "clocks": clocks}
+    step.close()
+    del step, host
+    torch.cuda.empty_cache()
+    return rec
+
+
+def oracle_one_thread(names):
+    """The oracle on ONE host thread (its OpenMP loops cut to a single thread), per workload, by the
+    same bounded-sample method as the reference arm: a child process of this script."""
+    out = {}
+    for name in names:
+        env = dict(os.environ, OMP_NUM_THREADS="1")
+        for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK"):
+            env.pop(k, None)
+        try:
+            r = subprocess.run([sys.executable, os.path.abspath(__file__), "--impl", "reference", "--config", name,
+                                "--steps", "1", "--warmup", "0", "--reference-visits", "2e7", "--reference-seqs", "1"],
+                               env=env, capture_output=True, text=True, timeout=240)
+            d = json.loads(r.stdout.strip().splitlines()[-1])
+            out[name] = {"value": d["value"], "unit": UNIT, "cores": d["cpu_baseline"]["cores"],
+                         "sample": d["cpu_baseline"]["sample"]}
+        except Exception as e:                                              # reported, never fatal for the GPU line
+            out[name] = {"error": repr(e)[:200]}
+    return out
 
 
 def run_ours(args, cfg):
@@ -332,6 +429,7 @@ def run_ours(args, cfg):
     ms_step = total_ms / args.steps
     part = lambda a, b: statistics.mean(ev[i][a].elapsed_time(ev[i][b]) for i in range(args.steps))  # noqa: E731
     ms_plan, ms_attn, ms_acc, ms_cmp = part(0, 1), part(1, 2), part(2, 3), part(3, 4)
+    ms_each = [ev[i][0].elapsed_time(ev[i][4]) for i in range(args.steps)]
     alen = step.accept_len.float().mean().item()
 
     def time_accept_variants():
@@ -452,16 +550,32 @@ def run_ours(args, cfg):
             dist.destroy_process_group()
         return
     peaks = measured_peaks()
-    a_bytes = attention_bytes_per_layer(cfg, plen)
-    a_flops = attention_flops_per_layer(cfg, plen)
-    attn_launch_s = ms_attn * 1e-3 / cfg.L
-    achieved = a_bytes / attn_launch_s / 1e9
+    sm_count = step_mod.sm_count(step)
+    lens = attention_lens(cfg, plen, ms_attn * 1e-3 / cfg.L, clocks, peaks, sm_count)
+    # the other workloads of the table (batch 1 shapes of the three model families, and one contemplate
+    # row per node), each with its own clock record; one GPU only, after the main workload's memory is gone
+    others = None
+    if world == 1 and not args.no_other_workloads and args.config == "batch32":
+        launches_main = args.steps * step.launches_per_step()
+        step.close()
+        for name in ("q", "k", "v", "ks", "vs", "out", "tl", "dl", "graphs"):
+            setattr(step, name, None)
+        torch.cuda.empty_cache()
+        others = {}
+        for name, temperature in (("llama3b", 1.0), ("llama8b", 1.0), ("qwen4b", 1.0), ("qwen4b", 0.0), ("batch32_2t", 1.0)):
+            key = name if temperature > 0 else name + "_greedy"
+            others[key] = time_other_workload(name, temperature, device, local, peaks)
+    else:
+        launches_main = args.steps * step.launches_per_step()
     sbytes = step_bytes(cfg, plen, alen)
     kname = "attention_tc_kernel" if step_mod.uses_tensor_core_path(cfg) else "attention_generic_kernel"
     cpu = oracle_sample(oracle_prepare(cfg)) if not args.no_cpu_baseline else None
+    cpu_1t = oracle_one_thread(("tiny", "llama3b")) if not args.no_cpu_baseline else None
+    tensor_bound = lens["bound"] == "tensor"
     line = {
         "metric": METRIC, "value": aggregate_value(world, args.steps, total_ms), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "ms_per_step_median": statistics.median(ms_each),
+        "ms_per_step_min": min(ms_each), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "layers": cfg.L, "heads": f"{cfg.Hq}q/{cfg.Hkv}kv", "head_dim": cfg.D,
                    "tree_rows": cfg.T, "contemplate_rows": cfg.C, "soft_prompt": cfg.S, "vocab": cfg.V,
@@ -477,25 +591,40 @@ def run_ours(args, cfg):
                    "accept_variants": accept_variants,
                    "step_bytes": sbytes, "step_gbs": sbytes / (ms_step * 1e-3) / 1e9,
                    "step_frac_of_hbm_roofline": sbytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                   "mean_accept_len": alen, "status_ok": status_ok, "spot_check_vs_oracle": checked},
-        "roofline": {"bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": profile_traffic(kname, inputs.CONFIGS[args.config].name),
-                     "peak_source": peaks["source"], "bytes_per_launch": a_bytes, "launch_ms": attn_launch_s * 1e3,
-                     "frac_of_nominal_8TBs": achieved / 8000.0,
-                     "tensor_tflops": a_flops / attn_launch_s / 1e12,
-                     "tensor_frac_of_bf16_peak": a_flops / attn_launch_s / 1e12 / peaks["bf16_tflops"]},
+                   "mcycles_per_step": None if not (clocks and clocks.get("sm_mhz")) else ms_step * 1e-3 * clocks["sm_mhz"],
+                   "mean_accept_len": alen, "status_ok": status_ok, "spot_check_vs_oracle": checked,
+                   "workloads": others},
+        # The dominant kernel (one attention launch = kernel + merge of the split partials) against the
+        # ceiling that binds at the measured peaks; the other ceiling's figures stand beside it.
+        "roofline": {"bound": lens["bound"], "kernel": kname,
+                     "achieved": lens["tensor_tflops"] if tensor_bound else lens["hbm_gbs"],
+                     "peak": peaks["bf16_tflops"] if tensor_bound else peaks["hbm_gbs"],
+                     "unit": "TFLOP/s" if tensor_bound else "GB/s",
+                     "frac": lens["frac_of_measured_bf16_sustained"] if tensor_bound else lens["frac_of_measured_hbm"],
+                     "traffic": profile_traffic(kname, inputs.CONFIGS[args.config].name),
+                     "peak_source": peaks["source"] + (" (sustained bf16 matmul rate: the kernel is timed inside a long step)"
+                                                       if tensor_bound else " (copy bandwidth)"),
+                     "hbm": {"achieved": lens["hbm_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": lens["frac_of_measured_hbm"], "frac_of_nominal_8TBs": lens["frac_of_nominal_8TBs"]},
+                     "tensor": {"achieved": lens["tensor_tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                "frac": lens["frac_of_measured_bf16_sustained"]},
+                     "floor_us": lens["floor_us"], "launch_ms": lens["launch_us"] * 1e-3,
+                     "bytes_per_launch": lens["bytes_per_launch"], "flops_per_launch": lens["flops_per_launch"],
+                     "key_tiles_per_launch": lens["key_tiles_per_launch"],
+                     "cycles_per_key_tile_per_sm": lens["cycles_per_key_tile_per_sm"]},
         "e2e": None if e2e is None else {
             "value": e2e[0], "unit": UNIT, "h2d_bytes_per_step": e2e[3], "d2h_bytes_per_step": e2e[4],
             "ms_per_step": e2e[1], "steps": e2e[2],
             "note": "per step: Q, the R rows' K/V (all layers), both logit matrices, tree arrays and uniforms "
                     "copied from pinned host memory on a copy stream that runs ahead of the compute stream (an event per layer); "
                     "results copied back; the prefix KV cache is resident state"},
-        "gpu_launches": args.steps * step.launches_per_step(),
+        "gpu_launches": launches_main,
         "clocks": clocks,
     }
     if cpu is not None:
         line["cpu_baseline"] = {"value": 1.0 / cpu["step_seconds_estimate"], "unit": UNIT, "cores": cpu["cores"],
-                                "kind": "oracle", "sample": cpu["sample"], "sample_seconds": cpu["sample_seconds"]}
+                                "kind": "oracle", "sample": cpu["sample"], "sample_seconds": cpu["sample_seconds"],
+                                "one_thread": cpu_1t}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -511,6 +640,10 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time kernel launches issued one by one from the host")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-other-workloads", action="store_true", help="time the chosen workload only")
+    ap.add_argument("--reference-visits", type=float, default=1.2e8,
+                    help="--impl reference: (row, key) pairs one timed sample of the oracle's attention visits")
+    ap.add_argument("--reference-seqs", type=int, default=8, help="--impl reference: sequences in one sample")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer count (profiling runs; named in config.workload)")
     ap.add_argument("--batch", type=int, default=0, help="cut the batch (profiling runs; named in config.workload)")
     args = ap.parse_args()

@@ -114,6 +114,11 @@ class VerifyStep:
         return 1 + attention_kernels_per_layer(self.cfg) * len(self.q) + 3
 
 
+def sm_count(step):
+    """SM count of the step's device (one attention CTA per SM)."""
+    return torch.cuda.get_device_properties(torch.device(step.dev)).multi_processor_count
+
+
 def uses_tensor_core_path(cfg):
     """Mirror of the library's dispatch rule: bf16, head dim 128, at most 4 query heads per KV head."""
     return cfg.kv_dtype == torch.bfloat16 and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
