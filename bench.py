@@ -24,6 +24,7 @@ sys.path.insert(0, ROOT)
 
 from paper_2603_08899_b200 import inputs  # noqa: E402
 
+ATTENTION_PATH = 0          # --attention-path
 METRIC = "verify_steps_per_sec"
 UNIT = "steps/s"
 
@@ -89,7 +90,9 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
 
 
-KERNEL_SOURCES = {"attention_tc_kernel": ("attn_tc.cu", "attn_tc.cuh"), "attention_generic_kernel": ("attn_generic.cu",)}
+KERNEL_SOURCES = {"attention_pair_kernel": ("attn_tc2.cu", "tc_walk.cuh", "tc_ptx.cuh", "attn_tc.cuh"),
+                  "attention_tc_kernel": ("attn_tc.cu", "tc_walk.cuh", "tc_ptx.cuh", "attn_tc.cuh"),
+                  "attention_generic_kernel": ("attn_generic.cu",)}
 
 
 def kernel_source_hash(kernel):
@@ -277,6 +280,9 @@ def build_workload(cfg, device, rank, temperature=1.0):
     tok = inputs.draft_tokens(cfg, parent, dl, temperature)
     u = inputs.uniforms(cfg)
     step = VerifyStep(cfg, n_slots, device=device)
+    if ATTENTION_PATH:
+        from paper_2603_08899_b200 import binding as cb
+        cb.confu_set_option(step.ctx, cb.OPT_ATTENTION_PATH, ATTENTION_PATH)
     step.bind(q, k, v, ks if cfg.S else None, vs if cfg.S else None, out, seq_start.to(device), plen.to(device),
               parent.to(device), owner.to(device) if cfg.C else None, tl, dl, tok.to(device), u.to(device))
     host = {"parent": parent, "owner": owner, "plen": plen, "seq_start": seq_start, "tok": tok, "u": u}
@@ -568,7 +574,7 @@ def run_ours(args, cfg):
     else:
         launches_main = args.steps * step.launches_per_step()
     sbytes = step_bytes(cfg, plen, alen)
-    kname = "attention_tc_kernel" if step_mod.uses_tensor_core_path(cfg) else "attention_generic_kernel"
+    kname = step_mod.attention_kernel_name(cfg)
     cpu = oracle_sample(oracle_prepare(cfg)) if not args.no_cpu_baseline else None
     cpu_1t = oracle_one_thread(("tiny", "llama3b")) if not args.no_cpu_baseline else None
     tensor_bound = lens["bound"] == "tensor"
@@ -641,12 +647,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-other-workloads", action="store_true", help="time the chosen workload only")
+    ap.add_argument("--attention-path", type=int, default=0,
+                    help="CONFU_ATTENTION_* for A/B runs: 0 the library's choice, 2 one CTA per SM, 3 CTA pairs")
     ap.add_argument("--reference-visits", type=float, default=1.2e8,
                     help="--impl reference: (row, key) pairs one timed sample of the oracle's attention visits")
     ap.add_argument("--reference-seqs", type=int, default=8, help="--impl reference: sequences in one sample")
     ap.add_argument("--layers", type=int, default=0, help="cut the layer count (profiling runs; named in config.workload)")
     ap.add_argument("--batch", type=int, default=0, help="cut the batch (profiling runs; named in config.workload)")
     args = ap.parse_args()
+    global ATTENTION_PATH
+    ATTENTION_PATH = args.attention_path
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = inputs.CONFIGS[args.config]
     cut = {k: v for k, v in (("L", args.layers), ("B", args.batch)) if v > 0}

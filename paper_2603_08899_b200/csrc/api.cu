@@ -42,6 +42,11 @@ size_t ws_total(const confu_ctx* ctx, const confu_dims* d)
 namespace confu {
 cudaError_t launch_bounded_wait(unsigned long long limit_ns, int32_t* status, cudaStream_t st);
 bool tc_attention_supported(const confu_dims& d);
+bool pair_attention_supported(const confu_dims& d, int sm_count);
+cudaError_t launch_attention_pair(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
+                                  const void* v_cache, int64_t n_slots, const SlotMap& map,
+                                  const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
+                                  void* partials, void* out, float* lse, int32_t* status, cudaStream_t st);
 cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
                                 const void* v_cache, int64_t n_slots, const SlotMap& map,
                                 const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
@@ -54,11 +59,11 @@ namespace {
 // (never _AUTO), or a negative error code when a forced path cannot take them.
 int resolve_attention_path(const confu_ctx* ctx, const confu_dims& d)
 {
-    const bool tc = tc_attention_supported(d);
+    const bool tc = tc_attention_supported(d), pair = pair_attention_supported(d, ctx->sm_count);
     switch (ctx->attention_path) {
         case CONFU_ATTENTION_GENERIC: return CONFU_ATTENTION_GENERIC;
         case CONFU_ATTENTION_TENSOR: return tc ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ERR_UNSUPPORTED;
-        case CONFU_ATTENTION_TENSOR_PAIR: return CONFU_ERR_UNSUPPORTED;
+        case CONFU_ATTENTION_TENSOR_PAIR: return pair ? (int)CONFU_ATTENTION_TENSOR_PAIR : (int)CONFU_ERR_UNSUPPORTED;
         default: return tc ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ATTENTION_GENERIC;
     }
 }
@@ -190,7 +195,10 @@ int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims, const int64_t* seq_s
     if (!plan) return CONFU_ERR_ARG;
     if (dims->B > 0 && (!prefix_len || !parent || (dims->C > 0 && !con_owner))) return CONFU_ERR_ARG;
     if (misaligned(plan)) return CONFU_ERR_ALIGN;
-    cudaError_t e = launch_plan(ctx, *dims, seq_start, prefix_len, parent, con_owner, plan, status, (cudaStream_t)stream);
+    const int path = resolve_attention_path(ctx, *dims);
+    if (path < 0) return path;
+    cudaError_t e = launch_plan(ctx, *dims, seq_start, prefix_len, parent, con_owner, plan, status,
+                                path == CONFU_ATTENTION_TENSOR_PAIR, (cudaStream_t)stream);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
 }
 
@@ -220,12 +228,16 @@ int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims, const void* q, 
     const void* use_plan = plan;
     if (!plan) {
         void* own_plan = ws + ws_plan_offset();
-        cudaError_t e = launch_plan(ctx, *dims, seq_start, prefix_len, parent, con_owner, own_plan, status, st);
+        cudaError_t e = launch_plan(ctx, *dims, seq_start, prefix_len, parent, con_owner, own_plan, status,
+                                    path == CONFU_ATTENTION_TENSOR_PAIR, st);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         use_plan = own_plan;
     }
     cudaError_t e;
-    if (path == CONFU_ATTENTION_TENSOR)
+    if (path == CONFU_ATTENTION_TENSOR_PAIR)
+        e = launch_attention_pair(ctx, *dims, q, k_cache, v_cache, n_slots, map, prefix_len, k_soft, v_soft,
+                                  use_plan, ws + ws_partial_offset(dims), out, lse, status, st);
+    else if (path == CONFU_ATTENTION_TENSOR)
         e = launch_attention_tc(ctx, *dims, q, k_cache, v_cache, n_slots, map, prefix_len, k_soft, v_soft,
                                 use_plan, ws + ws_partial_offset(dims), out, lse, status, st);
     else

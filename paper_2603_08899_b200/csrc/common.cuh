@@ -36,8 +36,8 @@ constexpr int kTileKeys = 128;                  // keys per attention tile (tens
 constexpr int kPairOverheadTiles = 4;
 struct PlanHeader {
     int32_t B, Hkv, T, C, S, R;
-    int32_t n_ctas;            // CTAs of the tensor-core attention launch (<= SM count)
-    int32_t pad;
+    int32_t n_ctas;            // work units of the tensor-core attention launch: CTAs (<= SM count) or CTA pairs
+    int32_t paired;            // 1: the runs are listed per CTA pair (two-SM kernel), 0: per CTA
     int64_t n_tiles;           // length N of the cost line
 };
 
@@ -207,7 +207,7 @@ __device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b)
 // launchers (defined in the .cu files)
 // ---------------------------------------------------------------------------
 cudaError_t launch_plan(const Ctx* ctx, const confu_dims& d, const int64_t* seq_start, const int32_t* prefix_len,
-                        const int32_t* parent, const int32_t* con_owner, void* plan, int32_t* status,
+                        const int32_t* parent, const int32_t* con_owner, void* plan, int32_t* status, bool paired,
                         cudaStream_t st);
 
 cudaError_t launch_attention_generic(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,

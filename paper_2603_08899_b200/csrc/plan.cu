@@ -8,7 +8,7 @@
 
 namespace confu {
 
-__global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, const int64_t* __restrict__ seq_start,
+__global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int units, int paired, const int64_t* __restrict__ seq_start,
                                                    const int32_t* __restrict__ prefix_len,
                                                    const int32_t* __restrict__ parent,
                                                    const int32_t* __restrict__ con_owner, void* plan_raw,
@@ -76,9 +76,9 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
         PlanHeader h;
         h.B = B; h.Hkv = d.Hkv; h.T = T; h.C = C; h.S = d.S; h.R = R;
         h.n_tiles = acc;
-        h.n_ctas = (int)(acc < (int64_t)sm_count ? acc : (int64_t)sm_count);
+        h.n_ctas = (int)(acc < (int64_t)units ? acc : (int64_t)units);
         if (h.n_ctas > kPlanMaxCtas) h.n_ctas = kPlanMaxCtas;
-        h.pad = 0;
+        h.paired = paired;
         *pv.hdr = h;
     }
     __syncthreads();
@@ -139,10 +139,12 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int sm_count, c
 }
 
 cudaError_t launch_plan(const Ctx* ctx, const confu_dims& d, const int64_t* seq_start, const int32_t* prefix_len,
-                        const int32_t* parent, const int32_t* con_owner, void* plan, int32_t* status,
+                        const int32_t* parent, const int32_t* con_owner, void* plan, int32_t* status, bool paired,
                         cudaStream_t st)
 {
-    plan_kernel<<<1, 256, 0, st>>>(d, ctx->sm_count, seq_start, prefix_len, parent, con_owner, plan, status);
+    // work units of the attention launch the plan is for: one CTA per SM, or one CTA pair per two SMs
+    const int units = paired ? ctx->sm_count / 2 : ctx->sm_count;
+    plan_kernel<<<1, 256, 0, st>>>(d, units, paired ? 1 : 0, seq_start, prefix_len, parent, con_owner, plan, status);
     return cudaGetLastError();
 }
 

@@ -124,6 +124,13 @@ def uses_tensor_core_path(cfg):
     return cfg.kv_dtype == torch.bfloat16 and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
 
 
+def attention_kernel_name(cfg):
+    """Mirror of the library's choice of attention kernel (CONFU_ATTENTION_AUTO)."""
+    if not uses_tensor_core_path(cfg):
+        return "attention_generic_kernel"
+    return "attention_tc_kernel"
+
+
 def attention_kernels_per_layer(cfg):
     """Tensor-core path: attention + split combine; generic path: one kernel."""
     return 2 if uses_tensor_core_path(cfg) else 1

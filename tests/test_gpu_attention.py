@@ -2,6 +2,7 @@
 import pytest
 import torch
 
+from paper_2603_08899_b200 import binding as cb
 from paper_2603_08899_b200 import inputs
 from tests import harness as H
 
@@ -59,12 +60,26 @@ CASES = {
 }
 
 
+def _takes_tensor_cores(cfg):
+    return cfg.kv_dtype == torch.bfloat16 and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
+
+
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("use_plan", [False, True])
-def test_attention_matches_oracle(gpu, name, use_plan):
+@pytest.mark.parametrize("path", ["auto", "one_cta_per_sm"])
+def test_attention_matches_oracle(gpu, name, use_plan, path):
+    """path auto: the library's own choice (CTA pairs with two-SM tensor-core instructions where the
+    dims allow, else one CTA per SM, else CUDA cores); one_cta_per_sm: the single-CTA tensor-core kernel
+    forced for every case it can take (it serves R <= 32 and odd SM counts in production)."""
     cfg = CASES[name]
+    if path != "auto" and not (_takes_tensor_cores(cfg) and cfg.R > 32):
+        pytest.skip("auto already runs this kernel")
     parent, owner, plen, seq_start, n_slots, t = H.setup_case(cfg)
-    out, lse, st = H.gpu_attention(gpu, cfg, t, seq_start, plen, parent, owner, n_slots, use_plan=use_plan)
+    gpu.set_path(cb.ATTENTION_AUTO if path == "auto" else cb.ATTENTION_TENSOR)
+    try:
+        out, lse, st = H.gpu_attention(gpu, cfg, t, seq_start, plen, parent, owner, n_slots, use_plan=use_plan)
+    finally:
+        gpu.set_path(cb.ATTENTION_AUTO)
     want, want_lse, want_st = H.oracle_attention(cfg, t, seq_start, plen, parent, owner)
     assert st.tolist() == want_st.tolist() == [0] * cfg.B
     H.assert_attention_close(out, lse, want, want_lse, cfg.kv_dtype, name)
@@ -99,8 +114,9 @@ def test_tree_rows_do_not_depend_on_soft_prompts_or_contemplate_rows(gpu):
     assert not torch.equal(a[:, cfg.T:], b[:, cfg.T:])
 
 
-def test_run_to_run_determinism(gpu):
-    cfg = CASES["bf16_g4_ragged_multi_tile"]
+@pytest.mark.parametrize("name", ["bf16_g4_ragged_multi_tile", "bf16_full_rows", "bf16_one_pair_130_parts"])
+def test_run_to_run_determinism(gpu, name):
+    cfg = CASES[name]
     parent, owner, plen, seq_start, n_slots, t = H.setup_case(cfg)
     a, la, _ = H.gpu_attention(gpu, cfg, t, seq_start, plen, parent, owner, n_slots)
     for _ in range(3):

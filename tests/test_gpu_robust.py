@@ -71,10 +71,16 @@ def test_packed_pool_with_poisoned_gaps(gpu, name, cfg):
     want, want_lse, _ = ref.tree_attention(t["q"], t["k_cache"], t["v_cache"], seq_start, plen, t["k_soft"],
                                            t["v_soft"], parent, owner)
     td = {k: (None if v is None else v.cuda()) for k, v in t.items()}
-    for use_plan in (False, True):
-        out, lse, st = H.gpu_attention(gpu, cfg, td, seq_start, plen, parent, owner, n_slots, use_plan=use_plan)
-        assert st.tolist() == [0] * cfg.B
-        H.assert_attention_close(out, lse, want, want_lse, cfg.kv_dtype, name)
+    paths = [cb.ATTENTION_AUTO] + ([cb.ATTENTION_TENSOR] if cfg.kv_dtype == torch.bfloat16 else [])
+    try:
+        for path in paths:
+            gpu.set_path(path)
+            for use_plan in (False, True):
+                out, lse, st = H.gpu_attention(gpu, cfg, td, seq_start, plen, parent, owner, n_slots, use_plan=use_plan)
+                assert st.tolist() == [0] * cfg.B
+                H.assert_attention_close(out, lse, want, want_lse, cfg.kv_dtype, f"{name} path {path}")
+    finally:
+        gpu.set_path(cb.ATTENTION_AUTO)
 
 
 @pytest.mark.parametrize("name,cfg", [
@@ -124,12 +130,18 @@ def test_a_malformed_tree_gives_zero_rows_on_every_path(gpu, cfg):
     bad = parent.clone()
     bad[1, 7] = 9                                         # parent index not below the node's own
     want, want_lse, want_st = H.oracle_attention(cfg, t, seq_start, plen, bad, owner)
-    for use_plan in (False, True):
-        out, lse, st = H.gpu_attention(gpu, cfg, t, seq_start, plen, bad, owner, n_slots, use_plan=use_plan)
-        assert st.tolist() == want_st.tolist() == [0, 1, 0]
-        assert (out[1] == 0).all() and (lse[1] == 0).all()
-        keep = [0, 2]
-        H.assert_attention_close(out[keep], lse[keep], want[keep], want_lse[keep], cfg.kv_dtype, "bad tree")
+    paths = [cb.ATTENTION_AUTO] + ([cb.ATTENTION_TENSOR] if cfg.kv_dtype == torch.bfloat16 else [])
+    try:
+        for path in paths:
+            gpu.set_path(path)
+            for use_plan in (False, True):
+                out, lse, st = H.gpu_attention(gpu, cfg, t, seq_start, plen, bad, owner, n_slots, use_plan=use_plan)
+                assert st.tolist() == want_st.tolist() == [0, 1, 0]
+                assert (out[1] == 0).all() and (lse[1] == 0).all()
+                keep = [0, 2]
+                H.assert_attention_close(out[keep], lse[keep], want[keep], want_lse[keep], cfg.kv_dtype, "bad tree")
+    finally:
+        gpu.set_path(cb.ATTENTION_AUTO)
 
 
 # ------------------------------------------------------------------ compaction with a bad path
@@ -272,14 +284,26 @@ def test_bounded_wait_gives_up_and_the_context_stays_usable(gpu):
 
 
 def test_attention_path_option(gpu):
-    cfg = _cfg(seed=81)
+    cfg = _cfg(T=30, C=10, seed=81)                       # more than 32 query rows: every path can take it
     parent, owner, plen, seq_start, n_slots, t = H.setup_case(cfg)
     want, want_lse, _ = H.oracle_attention(cfg, t, seq_start, plen, parent, owner)
     try:
-        for path in (cb.ATTENTION_GENERIC, cb.ATTENTION_TENSOR, cb.ATTENTION_AUTO):
+        for path in (cb.ATTENTION_GENERIC, cb.ATTENTION_TENSOR, cb.ATTENTION_TENSOR_PAIR, cb.ATTENTION_AUTO):
             gpu.set_path(path)
             out, lse, st = H.gpu_attention(gpu, cfg, t, seq_start, plen, parent, owner, n_slots)
             H.assert_attention_close(out, lse, want, want_lse, cfg.kv_dtype, f"path {path}")
+        # a plan only fits the path it was built for: the kernel refuses it with a status, nothing is computed
+        dims = H.dims_of(cfg)
+        gpu.set_path(cb.ATTENTION_TENSOR)
+        plan = torch.empty(cb.confu_plan_bytes(gpu.ctx, dims), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(cfg.B, dtype=torch.int32, device="cuda")
+        cb.confu_tree_plan(gpu.ctx, dims, seq_start.cuda(), plen.cuda(), parent.cuda(), owner.cuda(), plan, status)
+        gpu.set_path(cb.ATTENTION_TENSOR_PAIR)
+        out = torch.zeros_like(t["q"])
+        cb.confu_tree_attention(gpu.ctx, dims, t["q"], t["k_cache"], t["v_cache"], n_slots, seq_start.cuda(), plen.cuda(),
+                                t["k_soft"], t["v_soft"], None, None, plan, out, None, status)
+        torch.cuda.synchronize()
+        assert status.cpu().tolist() == [cb.ST_BAD_PLAN] * cfg.B
         # a forced tensor-core path refuses dims it cannot take
         gpu.set_path(cb.ATTENTION_TENSOR)
         cfg32 = _cfg(kv_dtype=torch.float32, seed=82)
