@@ -64,7 +64,15 @@ int resolve_attention_path(const confu_ctx* ctx, const confu_dims& d)
         case CONFU_ATTENTION_GENERIC: return CONFU_ATTENTION_GENERIC;
         case CONFU_ATTENTION_TENSOR: return tc ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ERR_UNSUPPORTED;
         case CONFU_ATTENTION_TENSOR_PAIR: return pair ? (int)CONFU_ATTENTION_TENSOR_PAIR : (int)CONFU_ERR_UNSUPPORTED;
-        default: return tc ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ATTENTION_GENERIC;
+        default: {
+            // The two-SM kernel wins where a (sequence, kv head, row group) is split over many work units
+            // (small batches: half as many, twice as long runs, half the partial results to merge); with
+            // more such pairs than units the one-CTA kernel is the faster one.
+            const int n_rg = (d.T + d.C + kGroupRows - 1) / kGroupRows;
+            const bool few_pairs = (int64_t)d.B * d.Hkv * n_rg <= ctx->sm_count / 2;
+            if (pair && few_pairs) return CONFU_ATTENTION_TENSOR_PAIR;
+            return tc ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ATTENTION_GENERIC;
+        }
     }
 }
 

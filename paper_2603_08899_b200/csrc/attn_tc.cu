@@ -232,20 +232,6 @@ __device__ void tail_role(SharedStorage& sh, const Params& prm, const PlanView& 
     if (have_prev) run_stage(0);
 }
 
-// max of 128 floats held as raw bits, as eight independent chains of three-input max
-__device__ __forceinline__ float max128(const uint32_t (&sv)[128])
-{
-    float a[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        a[k] = fmaxf(__uint_as_float(sv[16 * k]), __uint_as_float(sv[16 * k + 1]));
-#pragma unroll
-        for (int j = 2; j < 16; j += 2)
-            asm("max.f32 %0, %0, %1, %2;" : "+f"(a[k]) : "f"(__uint_as_float(sv[16 * k + j])), "f"(__uint_as_float(sv[16 * k + j + 1])));
-    }
-    return fmaxf(fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3])), fmaxf(fmaxf(a[4], a[5]), fmaxf(a[6], a[7])));
-}
-
 __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem, int t /*M tile*/)
 {
     const int lane_row = threadIdx.x & 127;                 // row of the M tile = TMEM lane

@@ -6,7 +6,7 @@
 // 128-key tile
 //     S = Q K^T      one M256 N128 K16 instruction per 16 head dims: each CTA supplies its 128 rows of
 //                    Q and 64 of the 128 keys, and receives its 128 rows of S in its own tensor memory
-//     P = exp2(S c - m)   two threads per row (64 keys each), bf16, into a tensor-memory buffer of its own
+//     P = exp2(S c - m)   one thread per row, bf16, into a tensor-memory buffer of its own
 //     O += P V       A = P from tensor memory, B = V: each CTA supplies 64 of the 128 head dims
 // so every K and V byte is fetched once per CTA pair, each SM reads half of the B operands from
 // its shared memory, and each SM carries ONE chain S -> softmax -> P -> P V.  With one chain per SM
@@ -14,10 +14,10 @@
 // P V of tile g, so the softmax warps always find their next S waiting and the tensor pipe works
 // on Q K^T while they compute exponentials.
 //
-// Roles per CTA (384 threads): warps 0-3 softmax of keys 0-63 of every tile, warps 4-7 of keys
-// 64-127 (the same 128 rows: each of the two threads of a row takes the row's maximum over all 128
-// scores itself and computes the weights of its 64; their sums meet through shared memory once per
-// run); warp 8 TMA producer (its own half of every tile, plain loads); warp 9 tensor
+// Roles per CTA (384 threads): warps 0-3 softmax of the even key tiles of the CTA's walk, warps 4-7
+// of the odd ones (the same 128 rows, one thread of each set per row: the two sets run half a tile
+// out of phase, so that one loads, masks and stores while the other keeps the exponential unit
+// busy; the row's reference maximum is handed from tile to tile through shared memory); warp 8 TMA producer (its own half of every tile, plain loads); warp 9 tensor
 // memory allocation and, in CTA 0, the one thread that issues every MMA of the pair; warp 10 the
 // relay: it waits for this CTA's loads, zeroes the rows of a V tile that lie past the sequence's
 // last slot, and tells CTA 0's issuing thread (remote mbarrier arrive) that this CTA's half of
@@ -33,7 +33,9 @@ namespace tc {
 namespace pair {
 
 constexpr int kThreads = 384;
-constexpr int kStages = 3;                          // ring of stages; stage g = [K of key tile g | V of key tile g - 1]
+constexpr int kStages = 4;                          // ring of stages; stage h = [K of key tile h | V of key tile h - kVLag]
+constexpr int kVLag = 2;                            // Q K^T runs about two tiles ahead of P V: a stage's K and V are used at about the same time
+constexpr int kQBufs = 1;                           // Q buffers (the next run's Q lands while this run's output rows are written)
 constexpr int kKHalf = 64 * 128;                    // this CTA's 64 keys x one 64-wide half of the head dim
 constexpr int kKBytes = 2 * kKHalf;                 // 16 KB
 constexpr int kVBytes = kTileKeys * 128;            // 128 keys x this CTA's 64 head dims: 16 KB
@@ -43,13 +45,14 @@ constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;   // S0 S1 | O | P0 P1 (
 constexpr float kRescaleThreshold = 8.f;
 
 struct SharedStorage {
-    alignas(1024) uint8_t q[2][kTileBytes];         // this CTA's 128 query rows, two 64-wide halves; double buffered
+    alignas(1024) uint8_t q[kQBufs][kTileBytes];    // this CTA's 128 query rows, two 64-wide halves
     alignas(1024) uint8_t kv[kStages][kStageBytes];
     alignas(16) float4 xpose[8][32 * 8];            // per softmax warp: 32 x 32 fp32 transpose tile of the epilogue
-    float xsum[2][128];                             // [key half][row]: the two threads of a row swap their sums at the end of a run
-    alignas(8) uint64_t q_full[2], q_ready[2], q_empty[2];
+    alignas(8) uint2 xref[2][128];                  // [set][row]: {tile tag, the row's reference maximum as of that tile}
+    float xsum[2][128], xm[2][128];                 // [set][row]: the two threads of a row swap sums and references at the end of a run
+    alignas(8) uint64_t q_full[kQBufs], q_ready[kQBufs], q_empty[kQBufs];
     uint64_t kv_full[kStages], kv_ready[kStages], kv_empty[kStages];
-    uint64_t s_full[2], p_full[2], o_done;
+    uint64_t s_full[2], s_free[2], p_full[2], o_done;
     uint64_t x_bar[4];                              // per pair of softmax warps (same rows): both have written xsum
     uint32_t tmem_base;
     int abort;
@@ -69,9 +72,12 @@ __device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
     return r;
 }
+// Arrival on a barrier of a CTA of the pair (an address from map_to_cta).  What the arrival orders is
+// tensor-memory traffic (tcgen05.wait / fence before it) and completed TMA copies, not generic-proxy
+// data: the default scope is enough, and a cluster-scope release costs ~1000 cycles here.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void store_remote_u32(uint32_t cluster_addr, uint32_t v)
 {
@@ -81,27 +87,26 @@ __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_try_wait_pair(uint64_t* bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
     return ok != 0;
 }
-// Bounded wait (cluster-scope acquire: the arrivals may come from the other CTA).  On expiry the abort
-// flags of both CTAs are raised.
+// Bounded wait.  On expiry the abort flags of both CTAs are raised.
 __device__ __forceinline__ bool wait_c(SharedStorage& sh, uint64_t* bar, uint32_t parity, unsigned long long limit_ns)
 {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (mbar_try_wait_pair(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     volatile int* abort = &sh.abort;
     for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (mbar_try_wait_pair(bar, parity)) return true;
         if ((it & 63u) == 0) {
             if (*abort) return false;
             if (global_ns() - t0 > limit_ns) {
@@ -112,6 +117,13 @@ __device__ __forceinline__ bool wait_c(SharedStorage& sh, uint64_t* bar, uint32_
         }
     }
 }
+__device__ __forceinline__ void raise_abort(SharedStorage& sh)
+{
+    *(volatile int*)&sh.abort = 1;
+    store_remote_u32(map_to_cta(&sh.abort, cluster_ctarank() ^ 1u), 1u);
+}
+constexpr uint32_t kSpinLimit = 1u << 22;           // polls of a shared-memory flag before a role gives up (~0.1 s)
+
 // The same for a whole warp: every lane leaves with the same answer, so that the warp-wide
 // instructions behind the wait (tcgen05.ld / st, __syncwarp) are never reached by a part of the warp.
 __device__ __forceinline__ bool wait_warp(SharedStorage& sh, uint64_t* bar, uint32_t parity, unsigned long long limit_ns)
@@ -154,6 +166,7 @@ constexpr uint32_t kIdescPV2 = kIdescQK2 | (1u << 16);
 struct TileRef {
     int g, z;                          // kv head, first slot (row) of the tile
     bool soft;
+    bool present;                      // false: no tile (before the first, behind the last)
 };
 
 // This CTA's half of every stage: 64 of the tile's keys (K, both 64-wide halves of the head dim) and 64
@@ -168,27 +181,34 @@ __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanVi
     uint32_t g = 0, seg = 0;
     const int R = prm.d.T + prm.d.C;
     const uint32_t q_box_bytes = 32u * prm.G * 128u;
-    TileRef prev = {0, 0, false};
-    bool have_prev = false;
+    TileRef hist[kVLag];               // the tiles of the last kVLag stages, oldest first: hist[0]'s V travels with this stage's K
+#pragma unroll
+    for (int i = 0; i < kVLag; ++i) hist[i].present = false;
     auto fill = [&](const TileRef* cur) -> bool {
         const uint32_t st = g % kStages;
+        const bool have_v = hist[0].present;
         if (!wait_c(sh, &sh.kv_empty[st], ((g / kStages) & 1) ^ 1, prm.wait_ns)) return false;
-        mbar_arrive_expect_tx(&sh.kv_full[st], (cur ? kKBytes : 0) + (have_prev ? kVBytes : 0));
+        mbar_arrive_expect_tx(&sh.kv_full[st], (cur ? kKBytes : 0) + (have_v ? kVBytes : 0));
         if (cur) {
             const CUtensorMap* m = cur->soft ? ks_map : k_map;
             tma_load_3d(sh.kv[st], m, &sh.kv_full[st], 0, cur->g, cur->z + 64 * (int)rank);
             tma_load_3d(sh.kv[st] + kKHalf, m, &sh.kv_full[st], 64, cur->g, cur->z + 64 * (int)rank);
         }
-        if (have_prev) {
-            const CUtensorMap* m = prev.soft ? vs_map : v_map;
-            tma_load_3d(sh.kv[st] + kKBytes, m, &sh.kv_full[st], 64 * (int)rank, prev.g, prev.z);
+        if (have_v) {
+            const CUtensorMap* m = hist[0].soft ? vs_map : v_map;
+            tma_load_3d(sh.kv[st] + kKBytes, m, &sh.kv_full[st], 64 * (int)rank, hist[0].g, hist[0].z);
         }
+#pragma unroll
+        for (int i = 0; i + 1 < kVLag; ++i) hist[i] = hist[i + 1];
+        if (cur) hist[kVLag - 1] = *cur;
+        else hist[kVLag - 1].present = false;
         ++g;
         return true;
     };
     while (w.next(s)) {
         for (int t = s.t0; t < s.t1; ++t) {
             TileRef cur;
+            cur.present = true;
             cur.g = s.g;
             cur.soft = t >= s.nkt;
             cur.z = cur.soft ? 0
@@ -196,19 +216,20 @@ __device__ void producer_role(SharedStorage& sh, const Params& prm, const PlanVi
                                         : (int)(s.slot0 + (int64_t)t * kTileKeys);
             if (!fill(&cur)) return;
             if (t == s.t0) {
-                const uint32_t qb = seg & 1;
-                if (!wait_c(sh, &sh.q_empty[qb], ((seg >> 1) & 1) ^ 1, prm.wait_ns)) return;
+                const uint32_t qb = seg % kQBufs;
+                if (!wait_c(sh, &sh.q_empty[qb], ((seg / kQBufs) & 1) ^ 1, prm.wait_ns)) return;
                 mbar_arrive_expect_tx(&sh.q_full[qb], 2u * q_box_bytes);
                 for (int kb = 0; kb < 2; ++kb)
                     tma_load_3d(sh.q[qb] + kb * kHalfTile, q_map, &sh.q_full[qb], kb * 64, s.g * prm.G,
                                 s.b * R + kGroupRows * s.rg + 32 * (int)rank);
             }
-            prev = cur;
-            have_prev = true;
         }
         ++seg;
     }
-    if (n_total > 0 && !fill(nullptr)) return;
+    // kVLag more stages: they carry the V tiles of the last key tiles (a stage may be empty when the
+    // whole walk is shorter than kVLag tiles)
+    for (int i = 0; i < (n_total > 0 ? kVLag : 0); ++i)
+        if (!fill(nullptr)) return;
 }
 
 // Waits for this CTA's loads of every stage (and of every run's Q), zeroes the rows of a sequence's
@@ -219,59 +240,73 @@ __device__ void relay_role(SharedStorage& sh, const Params& prm, const PlanView&
     Segment s;
     const int R = prm.d.T + prm.d.C, lane = threadIdx.x & 31;
     uint32_t g = 0, seg = 0;
-    int prev_valid = 0;
-    bool have_prev = false;
-    auto run_stage = [&](int cur_valid) -> bool {
+    int valid[kVLag];                  // ragged-row counts of the tiles of the last kVLag stages, oldest first (0: whole tile or no tile)
+#pragma unroll
+    for (int i = 0; i < kVLag; ++i) valid[i] = 0;
+    bool any = false;
+    auto run_stage = [&](bool have_cur, int cur_valid) -> bool {
         const uint32_t st = g % kStages;
         if (!wait_warp(sh, &sh.kv_full[st], (g / kStages) & 1, prm.wait_ns)) return false;
-        if (have_prev && prev_valid > 0) {
+        if (valid[0] > 0) {
             const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-            for (int off = prev_valid * 128 + lane * 16; off < kVBytes; off += 32 * 16)
+            for (int off = valid[0] * 128 + lane * 16; off < kVBytes; off += 32 * 16)
                 *reinterpret_cast<uint4*>(sh.kv[st] + kKBytes + off) = zero;
+            // generic-proxy stores that the other CTA's issuing threads hand to the tensor pipe: visible to the
+            // async proxy, and (this rare case only) ordered at cluster scope before the arrival
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("fence.acq_rel.cluster;" ::: "memory");
         }
         __syncwarp();
         if (lane == 0) mbar_arrive_remote(map_to_cta(&sh.kv_ready[st], 0));
+#pragma unroll
+        for (int i = 0; i + 1 < kVLag; ++i) valid[i] = valid[i + 1];
+        valid[kVLag - 1] = have_cur ? cur_valid : 0;
+        any = any || have_cur;
         ++g;
-        have_prev = true;
-        prev_valid = cur_valid;
         return true;
     };
     while (w.next(s)) {
         for (int tile = s.t0; tile < s.t1; ++tile) {
-            if (!run_stage(ragged_rows(s, tile, R))) return;
+            if (!run_stage(true, ragged_rows(s, tile, R))) return;
             if (tile == s.t0) {
-                const uint32_t qb = seg & 1;
-                if (!wait_warp(sh, &sh.q_full[qb], (seg >> 1) & 1, prm.wait_ns)) return;
+                const uint32_t qb = seg % kQBufs;
+                if (!wait_warp(sh, &sh.q_full[qb], (seg / kQBufs) & 1, prm.wait_ns)) return;
                 __syncwarp();
                 if (lane == 0) mbar_arrive_remote(map_to_cta(&sh.q_ready[qb], 0));
             }
         }
         ++seg;
     }
-    if (have_prev) run_stage(0);
+    for (int i = 0; i < (any ? kVLag : 0); ++i)
+        if (!run_stage(false, 0)) return;
 }
 
-// The one thread of the pair that issues tensor-core work (CTA 0).  Per stage g: Q K^T of key tile g
-// into S[g & 1], then -- once both CTAs have handed over P -- P V of key tile g - 1.
-__device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem)
+// Two threads of CTA 0 issue the tensor-core work of the pair, each waiting only for what its own
+// instructions need (the pipe takes instructions from both without loss), so that neither product
+// waits behind a wake-up that belongs to the other:
+//   qk_role   S[g & 1] = Q K^T of key tile g as soon as K has landed in both CTAs and the softmax
+//             warps of both have read the S buffer's previous contents (tile g - 2) into registers;
+//   pv_role   O += P V of key tile g as soon as V has landed and both CTAs have handed P over.
+// A stage [K of tile h | V of tile h - kVLag] is free again when both threads' instructions on it have completed.
+__device__ void qk_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem)
 {
     Walker w(pv, prm, blockIdx.x >> 1);
     Segment s;
     uint32_t g = 0, seg = 0;
-    const uint32_t q_lo[2] = {desc_lo(smem_u32(sh.q[0]), 16), desc_lo(smem_u32(sh.q[1]), 16)};
-    const uint32_t k_lo0 = desc_lo(smem_u32(sh.kv[0]), 16), v_lo0 = desc_lo(smem_u32(sh.kv[0] + kKBytes), 16);
+    uint32_t q_lo[kQBufs];
+    for (int i = 0; i < kQBufs; ++i) q_lo[i] = desc_lo(smem_u32(sh.q[i]), 16);
+    const uint32_t k_lo0 = desc_lo(smem_u32(sh.kv[0]), 16);
     constexpr uint32_t kStageStep = kStageBytes >> 4;
-    bool have_prev = false, prev_first = false, prev_last = false;
-
-    auto run_stage = [&](bool have_cur, bool cur_first, bool cur_last) -> bool {
-        const uint32_t st = g % kStages;
-        if (!wait_c(sh, &sh.kv_ready[st], (g / kStages) & 1, prm.wait_ns)) return false;
-        if (have_cur && cur_first && !wait_c(sh, &sh.q_ready[seg & 1], (seg >> 1) & 1, prm.wait_ns)) return false;
-        tc_fence_after();
-        if (have_cur) {
-            // S = Q K^T: 8 steps of 16 head dims; step i sits in 64-wide half i / 4 at byte 32 (i % 4) of the swizzled row
-            const uint32_t kl = k_lo0 + st * kStageStep, ql = q_lo[seg & 1];
+    while (w.next(s)) {
+        const int n_tiles = s.t1 - s.t0;
+        for (int j = 0; j < n_tiles; ++j, ++g) {
+            const uint32_t st = g % kStages;
+            if (!wait_c(sh, &sh.kv_ready[st], (g / kStages) & 1, prm.wait_ns)) return;
+            if (j == 0 && !wait_c(sh, &sh.q_ready[seg % kQBufs], (seg / kQBufs) & 1, prm.wait_ns)) return;
+            if (!wait_c(sh, &sh.s_free[g & 1], ((g >> 1) & 1) ^ 1, prm.wait_ns)) return;
+            tc_fence_after();
+            // 8 steps of 16 head dims; step i sits in 64-wide half i / 4 at byte 32 (i % 4) of the swizzled row
+            const uint32_t kl = k_lo0 + st * kStageStep, ql = q_lo[seg % kQBufs];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint32_t q_off = ((uint32_t)(i >> 2) * kHalfTile + (uint32_t)(i & 3) * 32u) >> 4;
@@ -279,75 +314,63 @@ __device__ void mma_role(SharedStorage& sh, const Params& prm, const PlanView& p
                 mma2_ss(tmem + kColS + (g & 1) * 128, ql + q_off, kl + k_off, kIdescQK2, i > 0 ? 1u : 0u);
             }
             commit_both(&sh.s_full[g & 1]);
-            if (cur_last) commit_both(&sh.q_empty[seg & 1]);       // every Q K^T of this run has been issued
+            commit_both(&sh.kv_empty[st]);
+            if (j + 1 == n_tiles) commit_both(&sh.q_empty[seg % kQBufs]);     // every Q K^T of this run has been issued
         }
-        if (have_prev) {
-            const uint32_t pb = (g - 1) & 1;
-            if (!wait_c(sh, &sh.p_full[pb], ((g - 1) >> 1) & 1, prm.wait_ns)) return false;
+        ++seg;
+    }
+    // the last kVLag stages carry no K tile: this thread has nothing to issue on them, but their release
+    // counts its arrival too (the softmax threads wait for it before they rescale O)
+    for (int i = 0; i < (g > 0 ? kVLag : 0); ++i, ++g) {
+        if (!wait_c(sh, &sh.kv_ready[g % kStages], (g / kStages) & 1, prm.wait_ns)) return;
+        commit_both(&sh.kv_empty[g % kStages]);
+    }
+}
+
+__device__ void pv_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem)
+{
+    Walker w(pv, prm, blockIdx.x >> 1);
+    Segment s;
+    uint32_t g = 0;
+    const uint32_t v_lo0 = desc_lo(smem_u32(sh.kv[0] + kKBytes), 16);
+    constexpr uint32_t kStageStep = kStageBytes >> 4;
+    // the first kVLag stages carry no V tile: this thread has nothing to wait for on them
+    for (int i = 0; i < kVLag; ++i) commit_both(&sh.kv_empty[i]);
+    while (w.next(s)) {
+        const int n_tiles = s.t1 - s.t0;
+        for (int j = 0; j < n_tiles; ++j, ++g) {
+            const uint32_t st = (g + kVLag) % kStages, pb = g & 1;      // V of tile g travels with K of tile g + kVLag
+            if (!wait_c(sh, &sh.kv_ready[st], ((g + kVLag) / kStages) & 1, prm.wait_ns)) return;
+            if (!wait_c(sh, &sh.p_full[pb], (g >> 1) & 1, prm.wait_ns)) return;
             tc_fence_after();
-            // O += P V: 8 steps of 16 keys (2048 B of the V tile and 8 tensor-memory columns of bf16 pairs each)
+            // 8 steps of 16 keys (2048 B of the V tile and 8 tensor-memory columns of bf16 pairs each)
             const uint32_t vl = v_lo0 + st * kStageStep;
 #pragma unroll
             for (int i = 0; i < 8; ++i)
                 mma2_ts(tmem + kColO, tmem + kColP + pb * 64 + i * 8, vl + i * (2048u >> 4), kIdescPV2,
-                        (prev_first && i == 0) ? 0u : 1u);
+                        (j == 0 && i == 0) ? 0u : 1u);
+            commit_both(&sh.kv_empty[st]);
+            if (j + 1 == n_tiles) commit_both(&sh.o_done);
         }
-        commit_both(&sh.kv_empty[st]);
-        if (have_prev && prev_last) commit_both(&sh.o_done);
-        ++g;
-        have_prev = have_cur;
-        prev_first = cur_first;
-        prev_last = cur_last;
-        return true;
-    };
-
-    while (w.next(s)) {
-        const int n_tiles = s.t1 - s.t0;
-        for (int j = 0; j < n_tiles; ++j)
-            if (!run_stage(true, j == 0, j + 1 == n_tiles)) return;
-        ++seg;
     }
-    if (have_prev) run_stage(false, false, false);
-}
-
-// max of 32 floats held as raw bits
-__device__ __forceinline__ float max32(const uint32_t (&sv)[32])
-{
-    float a[2];
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        a[k] = fmaxf(__uint_as_float(sv[16 * k]), __uint_as_float(sv[16 * k + 1]));
-#pragma unroll
-        for (int j = 2; j < 16; j += 2)
-            asm("max.f32 %0, %0, %1, %2;" : "+f"(a[k]) : "f"(__uint_as_float(sv[16 * k + j])), "f"(__uint_as_float(sv[16 * k + j + 1])));
-    }
-    return fmaxf(a[0], a[1]);
-}
-
-// max of 64 floats held as raw bits, as four independent chains of three-input max
-__device__ __forceinline__ float max64(const uint32_t (&sv)[64])
-{
-    float a[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        a[k] = fmaxf(__uint_as_float(sv[16 * k]), __uint_as_float(sv[16 * k + 1]));
-#pragma unroll
-        for (int j = 2; j < 16; j += 2)
-            asm("max.f32 %0, %0, %1, %2;" : "+f"(a[k]) : "f"(__uint_as_float(sv[16 * k + j])), "f"(__uint_as_float(sv[16 * k + j + 1])));
-    }
-    return fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
 }
 
 __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanView& pv, uint32_t tmem, uint32_t rank)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int half = warp >> 2, wq = warp & 3;               // which 64 keys of every tile; which 32 rows
+    // set 0 (warps 0-3) takes the even key tiles of the CTA's walk, set 1 (warps 4-7) the odd ones; at
+    // the end of a run set 0 writes head dims 0-63 of the output rows, set 1 head dims 64-127
+    const int set = warp >> 2, wq = warp & 3;
+    const int half = set;
     const int lane_row = wq * 32 + lane;                     // row of this CTA's 128 = tensor-memory lane
     const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
     const int G = prm.G, T = prm.d.T, R = prm.d.T + prm.d.C, S = prm.d.S, Hq = prm.d.Hq;
     const int hl = lane_row % G;
     const float c = prm.c;
-    const uint32_t p_full_leader[2] = {map_to_cta(&sh.p_full[0], 0), map_to_cta(&sh.p_full[1], 0)};
+    const uint32_t buf = (uint32_t)set;                      // S and P buffer of this set's tiles
+    const uint32_t p_full_leader = map_to_cta(&sh.p_full[buf], 0), s_free_leader = map_to_cta(&sh.s_free[buf], 0);
+    const uint32_t s_addr = tmem + lane_base + kColS + buf * 128, p_addr = tmem + lane_base + kColP + buf * 64;
+    const uint32_t ref_mine = smem_u32(&sh.xref[set][lane_row]), ref_theirs = smem_u32(&sh.xref[set ^ 1][lane_row]);
 
     Walker w(pv, prm, blockIdx.x >> 1);
     Segment s;
@@ -356,85 +379,99 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
         const int r = kGroupRows * s.rg + 32 * (int)rank + lane_row / G;      // query row of this thread in this run
         const bool row_valid = lane_row < 32 * G && r < R;
         const uint64_t mask = row_valid ? pv.mask[(size_t)s.b * kMaxRows + r] : 0ull;
-        float m_ref = -INFINITY, l = 0.f;
+        // this thread's share of the row's sum of weights, relative to the reference maximum m_mine
+        // (the row's reference as of the last tile this thread worked on)
+        float m_mine = -INFINITY, l = 0.f;
         for (int tile = s.t0; tile < s.t1; ++tile, ++g) {
-            const uint32_t buf = g & 1;
+            if ((g & 1u) != (uint32_t)set) continue;
             if (!wait_warp(sh, &sh.s_full[buf], (g >> 1) & 1, prm.wait_ns)) return;
             tc_fence_after();
-            // The row's maximum over all 128 scores (no exchange between the two threads of a row: both
-            // read everything), the weights only of this thread's 64.
-            const uint32_t s_base = tmem + lane_base + kColS + buf * 128;
-            uint32_t sv[64], ot[32];
-            tmem_ld32(s_base + (half ^ 1) * 64, ot);
-            tmem_ld32(s_base + half * 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-            tmem_ld32(s_base + half * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+            uint32_t sv[128];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(s_addr + q4 * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[q4 * 32]));
             tc_wait_ld();
+            // the scores sit in registers: the S buffer may take the tile after next
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(s_free_leader);
             const bool masked = tile >= s.nkt || (int64_t)(tile + 1) * kTileKeys > s.P;
-            uint64_t mine = ~0ull, theirs = ~0ull;
             if (masked) {
                 uint64_t lo, hi;
                 visible_bits(s, tile, R, T, S, r, row_valid, mask, lo, hi);
-                mine = half ? hi : lo;
-                theirs = half ? lo : hi;
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (!((theirs >> j) & 1ull)) ot[j] = 0xff800000u;        // -inf
-#pragma unroll
-                for (int j = 0; j < 64; ++j)
-                    if (!((mine >> j) & 1ull)) sv[j] = 0xff800000u;
-            }
-            float m_other = max32(ot);
-            tmem_ld32(s_base + (half ^ 1) * 64 + 32, ot);
-            const float m_own = max64(sv);
-            tc_wait_ld();
-            if (masked) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (!((theirs >> (32 + j)) & 1ull)) ot[j] = 0xff800000u;
-            }
-            m_other = fmaxf(m_other, max32(ot));
-            const float m_tile = fmaxf(m_own, m_other);
-            const float m_new = fmaxf(m_ref, m_tile * c);
-            if (tile == s.t0) {
-                m_ref = m_new;
-            } else {
-                const bool move = m_new - m_ref > kRescaleThreshold;         // false when both are -inf (NaN)
-                if (__any_sync(0xffffffffu, move)) {
-                    // O is being accumulated into by P V of the tile before: stage g's release says it is done
-                    if (!wait_warp(sh, &sh.kv_empty[g % kStages], (g / kStages) & 1, prm.wait_ns)) return;
-                    tc_fence_after();
-                    const float alpha = move ? ex2(m_ref - m_new) : 1.f;
-                    if (move) { m_ref = m_new; l *= alpha; }
-#pragma unroll
-                    for (int q4 = 0; q4 < 2; ++q4) {
-                        uint32_t ov[32];
-                        const uint32_t o_addr = tmem + lane_base + kColO + half * 64 + q4 * 32;
-                        tmem_ld32(o_addr, ov);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
-                        tmem_st32(o_addr, ov);
-                    }
+                for (int j = 0; j < 64; ++j) {
+                    if (!((lo >> j) & 1ull)) sv[j] = 0xff800000u;            // -inf
+                    if (!((hi >> j) & 1ull)) sv[64 + j] = 0xff800000u;
                 }
             }
+            const float m_tile = max128(sv) * c;
+            // The row's reference maximum is handed from tile to tile: the thread of the other set that
+            // worked on tile g - 1 published it (tagged with its tile; bounded spin), this one publishes
+            // the reference of tile g as soon as it is decided -- before any exponential.
+            float m_ref = m_tile, m_prev = -INFINITY;
+            bool move = false;
+            if (tile != s.t0) {
+                bool got = false;
+                for (uint32_t it = 0; it < kSpinLimit; ++it) {
+                    uint32_t tag, bits;
+                    asm volatile("ld.volatile.shared.v2.u32 {%0, %1}, [%2];" : "=r"(tag), "=r"(bits) : "r"(ref_theirs) : "memory");
+                    if (tag == g) { m_prev = __uint_as_float(bits); got = true; break; }
+                    if ((it & 1023u) == 1023u && *(volatile int*)&sh.abort) break;
+                }
+                if (!__all_sync(0xffffffffu, got)) { raise_abort(sh); return; }
+                move = m_tile - m_prev > kRescaleThreshold;                  // false when both are -inf (NaN)
+                m_ref = move ? m_tile : m_prev;
+            }
+            asm volatile("st.volatile.shared.v2.u32 [%0], {%1, %2};" ::"r"(ref_mine), "r"(g + 1), "r"(__float_as_uint(m_ref)) : "memory");
+            if (__any_sync(0xffffffffu, move)) {
+                // O is being accumulated into by P V of the tile before, whose V travelled in stage g - 1 + kVLag:
+                // that stage's release says it is done
+                if (!wait_warp(sh, &sh.kv_empty[(g - 1 + kVLag) % kStages], ((g - 1 + kVLag) / kStages) & 1, prm.wait_ns)) return;
+                tc_fence_after();
+                const float alpha = move ? ex2(m_prev - m_ref) : 1.f;       // O so far is relative to m_prev
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t ov[32];
+                    const uint32_t o_addr = tmem + lane_base + kColO + q4 * 32;
+                    tmem_ld32(o_addr, ov);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * alpha);
+                    tmem_st32(o_addr, ov);
+                }
+            }
+            // bring this thread's sum to the row's current reference
+            if (m_ref != m_mine) {
+                l = (m_mine == -INFINITY) ? 0.f : l * ex2(m_mine - m_ref);
+                m_mine = m_ref;
+            }
             const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-            uint32_t pk[32];
-            l += weights64(sv, c, neg_m, pk);
-            tmem_st32(tmem + lane_base + kColP + buf * 64 + half * 32, pk);
+            // the P buffer was last read by P V of tile g - 2, whose V travelled in stage g - 2 + kVLag
+            if (g >= 2 && !wait_warp(sh, &sh.kv_empty[(g - 2 + kVLag) % kStages], ((g - 2 + kVLag) / kStages) & 1, prm.wait_ns)) return;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t pk[32];
+                l += weights64(&sv[64 * hh], c, neg_m, pk);
+                tmem_st32(p_addr + 32 * hh, pk);
+            }
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_remote(p_full_leader[buf]);
+            if (lane == 0) mbar_arrive_remote(p_full_leader);
         }
-        // ---- end of the run: this thread's half of the row of O ----
+        // ---- end of the run: this thread's 64 head dims of the row of O ----
         if (!wait_warp(sh, &sh.o_done, seg & 1, prm.wait_ns)) return;
         tc_fence_after();
-        // the row's sum of weights: this thread's 64 keys plus the partner thread's (bounded wait, like every other)
-        sh.xsum[half][lane_row] = l;
+        // the row's sum of weights: the shares of the two threads of the row, each brought to the larger
+        // (= the final) reference maximum (bounded wait, like every other)
+        sh.xsum[set][lane_row] = l;
+        sh.xm[set][lane_row] = m_mine;
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.x_bar[wq]);
         if (!wait_warp(sh, &sh.x_bar[wq], seg & 1, prm.wait_ns)) return;
-        const float l_row = sh.xsum[0][lane_row] + sh.xsum[1][lane_row];
+        const float m_oth = sh.xm[set ^ 1][lane_row], l_oth = sh.xsum[set ^ 1][lane_row];
+        const float m_ref = fmaxf(m_mine, m_oth);
+        const float l_row = (m_mine == -INFINITY ? 0.f : l * ex2(m_mine - m_ref)) + (m_oth == -INFINITY ? 0.f : l_oth * ex2(m_oth - m_ref));
         const int h = s.g * G + hl;
         float4* xp = sh.xpose[warp];
         const bool whole = s.part_slot < 0;
@@ -522,21 +559,25 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
     const uint32_t rank = cluster_ctarank();
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kQBufs; ++i) {
             mbar_init(&sh.q_full[i], 1);
             mbar_init(&sh.q_ready[i], 2);
             mbar_init(&sh.q_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(&sh.s_full[i], 1);
-            mbar_init(&sh.p_full[i], 16);                   // one arrival per softmax warp of both CTAs
+            mbar_init(&sh.s_free[i], 8);                    // one arrival per softmax warp of a set, both CTAs
+            mbar_init(&sh.p_full[i], 8);
         }
         for (int i = 0; i < kStages; ++i) {
             mbar_init(&sh.kv_full[i], 1);
             mbar_init(&sh.kv_ready[i], 2);                  // the relay warps of both CTAs
-            mbar_init(&sh.kv_empty[i], 1);
+            mbar_init(&sh.kv_empty[i], 2);                  // the commits of both issuing threads
         }
         mbar_init(&sh.o_done, 1);
         for (int i = 0; i < 4; ++i) mbar_init(&sh.x_bar[i], 2);
         sh.abort = 0;
+        for (int i = 0; i < 2 * 128; ++i) (&sh.xref[0][0])[i] = make_uint2(0u, 0u);            // tag 0: no tile
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -554,13 +595,20 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
     const uint32_t tmem = sh.tmem_base;
 
     if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         softmax_role(sh, prm, pv, tmem, rank);
     } else if (warp == 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
         if ((threadIdx.x & 31) == 0) producer_role(sh, prm, pv, rank, &q_map, &k_map, &v_map, &ks_map, &vs_map);
     } else if (warp == 9) {
-        if ((threadIdx.x & 31) == 0 && rank == 0) mma_role(sh, prm, pv, tmem);
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        if ((threadIdx.x & 31) == 0 && rank == 0) qk_role(sh, prm, pv, tmem);
     } else if (warp == 10) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
         relay_role(sh, prm, pv);
+    } else if (warp == 11) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        if ((threadIdx.x & 31) == 0 && rank == 0) pv_role(sh, prm, pv, tmem);
     }
     __syncwarp();
     // ---- teardown ----

@@ -87,6 +87,20 @@ __device__ __forceinline__ void visible_bits(const Segment& s, int t, int R, int
     hi = (uint64_t)(v >> 64);
 }
 
+// max of 128 floats held as raw bits, as eight independent chains of three-input max
+__device__ __forceinline__ float max128(const uint32_t (&sv)[128])
+{
+    float a[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        a[k] = fmaxf(__uint_as_float(sv[16 * k]), __uint_as_float(sv[16 * k + 1]));
+#pragma unroll
+        for (int j = 2; j < 16; j += 2)
+            asm("max.f32 %0, %0, %1, %2;" : "+f"(a[k]) : "f"(__uint_as_float(sv[16 * k + j])), "f"(__uint_as_float(sv[16 * k + j + 1])));
+    }
+    return fmaxf(fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3])), fmaxf(fmaxf(a[4], a[5]), fmaxf(a[6], a[7])));
+}
+
 // exp2(s*c - m) of 64 scores -> 32 packed bf16 pairs; returns their fp32 sum
 __device__ __forceinline__ float weights64(const uint32_t* sv, float c, float neg_m, uint32_t (&pk)[32])
 {

@@ -128,7 +128,10 @@ def attention_kernel_name(cfg):
     """Mirror of the library's choice of attention kernel (CONFU_ATTENTION_AUTO)."""
     if not uses_tensor_core_path(cfg):
         return "attention_generic_kernel"
-    return "attention_tc_kernel"
+    n_rg = (cfg.T + cfg.C + 63) // 64
+    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count if torch.cuda.is_available() else 148
+    few_pairs = cfg.B * cfg.Hkv * n_rg <= sms // 2
+    return "attention_pair_kernel" if (cfg.T + cfg.C > 32 and few_pairs) else "attention_tc_kernel"
 
 
 def attention_kernels_per_layer(cfg):

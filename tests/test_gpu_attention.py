@@ -66,16 +66,18 @@ def _takes_tensor_cores(cfg):
 
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("use_plan", [False, True])
-@pytest.mark.parametrize("path", ["auto", "one_cta_per_sm"])
+@pytest.mark.parametrize("path", ["auto", "one_cta_per_sm", "cta_pairs"])
 def test_attention_matches_oracle(gpu, name, use_plan, path):
-    """path auto: the library's own choice (CTA pairs with two-SM tensor-core instructions where the
-    dims allow, else one CTA per SM, else CUDA cores); one_cta_per_sm: the single-CTA tensor-core kernel
-    forced for every case it can take (it serves R <= 32 and odd SM counts in production)."""
+    """path auto: the library's own choice (CUDA cores, one CTA per SM with tcgen05, or CTA pairs with
+    the two-SM instructions, by dims and batch size); the two tensor-core kernels are also forced, each
+    for every case it can take."""
     cfg = CASES[name]
-    if path != "auto" and not (_takes_tensor_cores(cfg) and cfg.R > 32):
-        pytest.skip("auto already runs this kernel")
+    if path == "one_cta_per_sm" and not _takes_tensor_cores(cfg):
+        pytest.skip("not a tensor-core case")
+    if path == "cta_pairs" and not (_takes_tensor_cores(cfg) and cfg.R > 32):
+        pytest.skip("the two-SM kernel takes more than 32 query rows")
     parent, owner, plen, seq_start, n_slots, t = H.setup_case(cfg)
-    gpu.set_path(cb.ATTENTION_AUTO if path == "auto" else cb.ATTENTION_TENSOR)
+    gpu.set_path({"auto": cb.ATTENTION_AUTO, "one_cta_per_sm": cb.ATTENTION_TENSOR, "cta_pairs": cb.ATTENTION_TENSOR_PAIR}[path])
     try:
         out, lse, st = H.gpu_attention(gpu, cfg, t, seq_start, plen, parent, owner, n_slots, use_plan=use_plan)
     finally:

@@ -71,7 +71,8 @@ def test_packed_pool_with_poisoned_gaps(gpu, name, cfg):
     want, want_lse, _ = ref.tree_attention(t["q"], t["k_cache"], t["v_cache"], seq_start, plen, t["k_soft"],
                                            t["v_soft"], parent, owner)
     td = {k: (None if v is None else v.cuda()) for k, v in t.items()}
-    paths = [cb.ATTENTION_AUTO] + ([cb.ATTENTION_TENSOR] if cfg.kv_dtype == torch.bfloat16 else [])
+    paths = [cb.ATTENTION_AUTO] + ([cb.ATTENTION_TENSOR] if cfg.kv_dtype == torch.bfloat16 else []) + \
+        ([cb.ATTENTION_TENSOR_PAIR] if cfg.kv_dtype == torch.bfloat16 and cfg.R > 32 else [])
     try:
         for path in paths:
             gpu.set_path(path)
@@ -130,7 +131,8 @@ def test_a_malformed_tree_gives_zero_rows_on_every_path(gpu, cfg):
     bad = parent.clone()
     bad[1, 7] = 9                                         # parent index not below the node's own
     want, want_lse, want_st = H.oracle_attention(cfg, t, seq_start, plen, bad, owner)
-    paths = [cb.ATTENTION_AUTO] + ([cb.ATTENTION_TENSOR] if cfg.kv_dtype == torch.bfloat16 else [])
+    paths = [cb.ATTENTION_AUTO] + ([cb.ATTENTION_TENSOR] if cfg.kv_dtype == torch.bfloat16 else []) + \
+        ([cb.ATTENTION_TENSOR_PAIR] if cfg.kv_dtype == torch.bfloat16 and cfg.R > 32 else [])
     try:
         for path in paths:
             gpu.set_path(path)
