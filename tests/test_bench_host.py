@@ -50,8 +50,9 @@ def test_profile_traffic_is_dropped_when_the_kernel_source_changed(tmp_path, mon
     monkeypatch.setattr(bench, "ROOT", str(tmp_path))
     os.makedirs(tmp_path / "profiles")
     os.makedirs(tmp_path / "paper_2603_08899_b200" / "csrc")
+    for name in bench.KERNEL_SOURCES["attention_tc_kernel"]:
+        (tmp_path / "paper_2603_08899_b200" / "csrc" / name).write_text("// h1\n")
     (tmp_path / "paper_2603_08899_b200" / "csrc" / "attn_tc.cu").write_text("// v1\n")
-    (tmp_path / "paper_2603_08899_b200" / "csrc" / "attn_tc.cuh").write_text("// h1\n")
     sha = bench.kernel_source_hash("attention_tc_kernel")
     (tmp_path / "profiles" / "attention_tc_kernel_batch32_L1.md").write_text(
         f"x\ntraffic_bytes_per_launch: 123\nkernel_source_sha256_16: {sha}\n")
