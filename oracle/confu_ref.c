@@ -536,6 +536,60 @@ int confu_ref_tree_accept_match(int32_t B, int32_t T, int32_t C, int32_t V, int3
 }
 
 /* ------------------------------------------------------------------ */
+/* 8-bit floating point cache entries (E4M3)                           */
+/* ------------------------------------------------------------------ */
+/*
+ * E4M3 as the OCP 8-bit floating point specification defines it: 1 sign bit, 4 exponent bits (bias
+ * 7), 3 mantissa bits; exponent 0 is subnormal (mantissa * 2^-9); there are no infinities; S.1111.111
+ * is NaN; the largest magnitude is S.1111.110 = 448.
+ */
+static double e4m3_value(uint8_t c)
+{
+    const int sign = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m, -9);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+int confu_ref_e4m3_decode(const uint8_t* src, int64_t n, double* dst)
+{
+    if (!src || !dst || n < 0) return -1;
+    for (int64_t i = 0; i < n; ++i) dst[i] = e4m3_value(src[i]);
+    return 0;
+}
+
+/*
+ * The quantisation a cache entry goes through when it is written: x / scale in SINGLE precision (the
+ * precision the decision is taken in on the device too), rounded to the nearest E4M3 value, ties to
+ * the value with an even mantissa, magnitudes beyond 448 saturating to 448; NaN stays NaN.
+ * Written as a search over the 127 non-negative finite codes: no bit tricks to get wrong.
+ */
+static uint8_t e4m3_code(float y)
+{
+    if (isnan(y)) return 0x7f;
+    const uint8_t sign = signbit(y) ? 0x80 : 0x00;
+    const double a = fabs((double)y);
+    if (a >= 448.0) return (uint8_t)(sign | 0x7e);
+    uint8_t best = 0;
+    double best_d = INFINITY;
+    for (int c = 0; c <= 0x7e; ++c) {
+        const double d = fabs(e4m3_value((uint8_t)c) - a);
+        /* codes ascend with their values: of two equally near neighbours the even code is the one with the even mantissa */
+        if (d < best_d || (d == best_d && (c & 1) == 0)) { best_d = d; best = (uint8_t)c; }
+    }
+    return (uint8_t)(sign | best);
+}
+
+int confu_ref_e4m3_encode(const float* src, float scale, int64_t n, uint8_t* dst)
+{
+    if (!src || !dst || n < 0 || !(scale > 0.0f)) return -1;
+    for (int64_t i = 0; i < n; ++i) dst[i] = e4m3_code(src[i] / scale);
+    return 0;
+}
+
+/* ------------------------------------------------------------------ */
 /* compaction                                                          */
 /* ------------------------------------------------------------------ */
 int confu_ref_kv_compact(int32_t B, int32_t n_layers, int64_t row_bytes,

@@ -17,7 +17,9 @@
  * closeness records of the acceptance walks (ratio_margin, resample_margin,
  * draw_margin, alt_token and the two "within 1e-5" counters) are pinned by
  * hand-computed cases, by cases planted inside and just outside the 1e-5 band,
- * and by exact-rational walks.
+ * and by exact-rational walks.  The E4M3 decode is pinned against a library conversion of all 256
+ * codes and against hand-written values; the encode against the library conversion on random
+ * values, hand-written ties, the saturation bound and the subnormal range.
  * The whole verify step on synthetic inputs has no published numbers:
  * beyond those pins, end-to-end parity is unpinned.
  *
@@ -184,6 +186,19 @@ int confu_ref_con_embedding(int32_t B, int32_t H_in, int32_t H_out, int32_t n_ex
 
 /* number of OpenMP threads the oracle will use */
 int confu_ref_num_threads(void);
+
+/*
+ * 8-bit floating point (E4M3) cache entries.  A cache that holds K and V as E4M3 bytes with one
+ * fp32 scale per KV head stands for the values  decode(byte) * scale[head]  -- exactly: the
+ * attention of such a cache is the definition above applied to those values (widened to double;
+ * the product of a 4-bit significand and an fp32 scale is exact in double).  The paper has no cache
+ * format; this is the 8-bit format serving engines use for KV caches.
+ * decode: dst[i] = value of code src[i] (NaN for S.1111.111).
+ * encode: dst[i] = nearest E4M3 code of src[i] / scale, the quotient taken in single precision,
+ *         ties to the even mantissa, saturating at +-448; scale > 0.
+ */
+int confu_ref_e4m3_decode(const uint8_t* src, int64_t n, double* dst);
+int confu_ref_e4m3_encode(const float* src, float scale, int64_t n, uint8_t* dst);
 
 #ifdef __cplusplus
 }

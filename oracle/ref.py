@@ -38,7 +38,7 @@ def lib():
         _lib.confu_ref_num_threads.restype = C.c_int
         for name in ("confu_ref_tree_attention", "confu_ref_tree_attention_rows",
                      "confu_ref_tree_accept", "confu_ref_tree_accept_match", "confu_ref_kv_compact",
-                     "confu_ref_con_embedding"):
+                     "confu_ref_con_embedding", "confu_ref_e4m3_decode", "confu_ref_e4m3_encode"):
             getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -214,3 +214,47 @@ def con_embedding(hidden, router_w, router_b, experts, k_expert, renormalize=Fal
     if rc != 0:
         raise ValueError("confu_ref_con_embedding: bad argument")
     return out, sel, gate, gap
+
+
+def e4m3_decode(codes):
+    """uint8 tensor of E4M3 codes -> fp64 values (same shape)."""
+    c = codes.contiguous()
+    assert c.dtype == torch.uint8 and c.device.type == "cpu"
+    out = torch.empty(c.shape, dtype=torch.float64)
+    if lib().confu_ref_e4m3_decode(_p(c), C.c_int64(c.numel()), _p(out)) != 0:
+        raise ValueError("confu_ref_e4m3_decode: bad argument")
+    return out
+
+
+def e4m3_encode(x, scale):
+    """fp32 tensor -> uint8 E4M3 codes of x / scale (one scale for the whole tensor)."""
+    x = x.to(torch.float32).contiguous()
+    out = torch.empty(x.shape, dtype=torch.uint8)
+    if lib().confu_ref_e4m3_encode(_p(x), C.c_float(float(scale)), C.c_int64(x.numel()), _p(out)) != 0:
+        raise ValueError("confu_ref_e4m3_encode: bad argument")
+    return out
+
+
+def quantize_cache(x, scale):
+    """[n_slots, Hkv, D] bf16/fp32 rows -> E4M3 codes with one scale per KV head (scale: [Hkv] fp32)."""
+    out = torch.empty(x.shape, dtype=torch.uint8)
+    for g in range(x.shape[1]):
+        out[:, g] = e4m3_encode(x[:, g].float(), float(scale[g]))
+    return out
+
+
+def dequantize_cache(codes, scale):
+    """E4M3 codes [n, Hkv, D] and per-head scales [Hkv] -> the fp64 values the cache stands for."""
+    v = e4m3_decode(codes)
+    return v * scale.to(torch.float64).view(1, -1, 1)
+
+
+def tree_attention_fp8(q, k_codes, v_codes, k_scale, v_scale, seq_start, prefix_len, ks_codes, vs_codes, parent,
+                       con_owner, sm_scale=0.0):
+    """Attention over an E4M3 cache: the definition applied to the values the cache stands for
+    (bytes and scales widened exactly); q is widened exactly as well."""
+    k = dequantize_cache(k_codes, k_scale)
+    v = dequantize_cache(v_codes, v_scale)
+    ks = None if ks_codes is None else dequantize_cache(ks_codes, k_scale)
+    vs = None if vs_codes is None else dequantize_cache(vs_codes, v_scale)
+    return tree_attention(q.to(torch.float64), k, v, seq_start, prefix_len, ks, vs, parent, con_owner, sm_scale=sm_scale)

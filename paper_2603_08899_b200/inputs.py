@@ -201,6 +201,15 @@ def layer_tensors(cfg: VerifyConfig, layer: int, n_slots: int, device="cpu", tre
     return {"q": q, "k_cache": k, "v_cache": v, "k_soft": ks, "v_soft": vs}
 
 
+def fp8_scales(cfg: VerifyConfig, layer: int):
+    """Per-KV-head fp32 scales of an E4M3 cache: the N(0,1) entries are mapped so that about 6 standard
+    deviations reach the format's largest value (448), jittered per head and layer."""
+    rng = _rng(cfg, 300 + layer)
+    k = (6.0 / 448.0) * (1.0 + 0.2 * rng.random(cfg.Hkv))
+    v = (6.0 / 448.0) * (1.0 + 0.2 * rng.random(cfg.Hkv))
+    return torch.from_numpy(k.astype(np.float32)), torch.from_numpy(v.astype(np.float32))
+
+
 def logits(cfg: VerifyConfig, device="cpu"):
     """target, draft logits [B,T,V] in cfg.logit_dtype."""
     g = _gen(cfg, 7, device)
