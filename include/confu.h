@@ -77,7 +77,7 @@ enum {
     CONFU_ST_BAD_PLAN = 10       /* confu_tree_attention: the plan was built for another attention path */
 };
 
-enum { CONFU_BF16 = 0, CONFU_F32 = 1 };
+enum { CONFU_BF16 = 0, CONFU_F32 = 1, CONFU_FP8_E4M3 = 2 };   /* FP8: cache entries only, see confu_set_kv_scales */
 
 #define CONFU_MAX_TREE  64      /* T: tree rows (one 64-bit ancestor word per row) */
 #define CONFU_MAX_ROWS  128     /* R = T + C, with C <= 64: covers one contemplate row per node (R = 2T) */
@@ -90,7 +90,8 @@ typedef struct {
     int32_t D;          /* head dim: 64 or 128 */
     int32_t T, C;       /* tree rows (root included), contemplate rows */
     int32_t S;          /* soft-prompt KV entries, shared by all sequences (0 allowed) */
-    int32_t kv_dtype;   /* CONFU_BF16 | CONFU_F32: type of q, caches, soft KV and out */
+    int32_t kv_dtype;   /* CONFU_BF16 | CONFU_F32: type of q, caches, soft KV and out;
+                           CONFU_FP8_E4M3: caches and soft KV are E4M3 bytes, q and out are bf16 */
     float   sm_scale;   /* 0 -> D^-1/2 */
 } confu_dims;
 
@@ -146,6 +147,24 @@ int confu_set_option(confu_ctx* ctx, int32_t option, int64_t value);
  * (device int32) and returns.  The context stays usable.
  */
 int confu_selftest_bounded_wait(confu_ctx* ctx, int64_t limit_ns, int32_t* status, void* stream);
+
+/*
+ * 8-bit floating point caches (kv_dtype = CONFU_FP8_E4M3; the paper has no cache format: this is
+ * the 8-bit KV cache of serving engines, a bandwidth and tensor-rate lever for the verification
+ * forward of Sec. 3.1).  A cache entry is an E4M3 byte (OCP 8-bit floating point: 1-4-3, bias 7, no
+ * infinities, largest magnitude 448) and stands for  code * scale[kv head] : k_scale, v_scale are
+ * DEVICE fp32 arrays of Hkv entries, read by every later call of this context until they are set
+ * again (set them per layer if the layers have scales of their own); the soft-prompt K/V use the
+ * same scales.  With these dims
+ *   - confu_tree_attention computes the attention of the values the cache stands for; q and out are
+ *     bf16; inside, Q (per row) and the softmax weights are rounded to E4M3 for the tensor cores
+ *     (kind::f8f6f4), accumulation is fp32 -- see the tolerance in the tests.  D = 128, Hq/Hkv <= 4,
+ *     S <= 128; CONFU_ERR_UNSUPPORTED otherwise, or without scales;
+ *   - confu_kv_append takes bf16 rows and stores  e4m3(row / scale)  (quotient in fp32, round to
+ *     nearest even, saturating at 448);
+ *   - confu_kv_compact moves bytes as for any other type.
+ */
+int confu_set_kv_scales(confu_ctx* ctx, const float* k_scale, const float* v_scale);
 
 const char* confu_status_string(int code);      /* host return codes and device status codes */
 const char* confu_last_cuda_error(const confu_ctx* ctx);

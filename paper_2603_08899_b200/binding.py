@@ -16,7 +16,7 @@ MAX_TREE = 64
 MAX_ROWS = 128
 MAX_DEPTH = 63
 ACCEPT_LAZY = 0x100          # or-ed into sibling_mode: row statistics on demand
-BF16, F32 = 0, 1
+BF16, F32, FP8_E4M3 = 0, 1, 2
 OK = 0
 OPT_ATTENTION_PATH, OPT_WAIT_LIMIT_NS = 1, 2
 ATTENTION_AUTO, ATTENTION_GENERIC, ATTENTION_TENSOR, ATTENTION_TENSOR_PAIR = 0, 1, 2, 3
@@ -27,7 +27,7 @@ EXPORTS = [
     "confu_last_cuda_error", "confu_plan_bytes", "confu_tree_plan", "confu_tree_attention",
     "confu_accept_workspace_bytes", "confu_tree_accept", "confu_kv_compact", "confu_kv_append",
     "confu_tree_accept_static_max_rows", "confu_tree_accept_static", "confu_set_paging",
-    "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_selftest_bounded_wait",
+    "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_selftest_bounded_wait", "confu_set_kv_scales",
 ]
 
 
@@ -55,7 +55,7 @@ def lib():
         L.confu_last_cuda_error.restype = C.c_char_p
         for n in ("confu_create", "confu_destroy", "confu_set_workspace", "confu_tree_plan", "confu_tree_attention",
                   "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static", "confu_set_paging",
-                  "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_selftest_bounded_wait"):
+                  "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_selftest_bounded_wait", "confu_set_kv_scales"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -89,7 +89,7 @@ def _check(fn, rc, ctx=None):
 
 
 def dtype_code(dt):
-    return {torch.bfloat16: BF16, torch.float32: F32}[dt]
+    return {torch.bfloat16: BF16, torch.float32: F32, torch.uint8: FP8_E4M3, torch.float8_e4m3fn: FP8_E4M3}[dt]
 
 
 def make_dims(B, Hq, Hkv, D, T, Cn, S, dtype, sm_scale=0.0):
@@ -119,6 +119,11 @@ def confu_set_workspace(ctx, tensor):
 def confu_set_paging(ctx, block_table, max_pages=0):
     """block_table: int32 CUDA tensor [B, max_pages] (kept alive by the caller), or None for packed pools."""
     _check("confu_set_paging", lib().confu_set_paging(ctx, _ptr(block_table), C.c_int32(max_pages)))
+
+
+def confu_set_kv_scales(ctx, k_scale, v_scale):
+    """k_scale, v_scale: fp32 CUDA tensors [Hkv] (kept alive by the caller), or None, None."""
+    _check("confu_set_kv_scales", lib().confu_set_kv_scales(ctx, _ptr(k_scale), _ptr(v_scale)))
 
 
 def confu_set_option(ctx, option, value):

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libconfu.so")
-SOURCES = ["api.cu", "plan.cu", "attn_generic.cu", "attn_tc.cu", "attn_tc2.cu", "combine.cu", "accept.cu", "accept_static.cu", "compact.cu", "moe.cu", "selftest.cu"]
+SOURCES = ["api.cu", "plan.cu", "attn_generic.cu", "attn_tc.cu", "attn_tc2.cu", "attn_fp8.cu", "combine.cu", "accept.cu", "accept_static.cu", "compact.cu", "moe.cu", "selftest.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "attn_tc.cuh"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(CSRC, "tc_walk.cuh"), os.path.join(ROOT, "include", "confu.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",

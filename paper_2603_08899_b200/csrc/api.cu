@@ -17,7 +17,8 @@ int check_dims(const confu_dims* d)
     if (d->B < 0 || d->Hq <= 0 || d->Hkv <= 0 || d->T <= 0 || d->C < 0 || d->S < 0) return CONFU_ERR_SHAPE;
     if (d->Hq % d->Hkv != 0) return CONFU_ERR_SHAPE;
     if (d->D != 64 && d->D != 128) return CONFU_ERR_SHAPE;
-    if (d->kv_dtype != CONFU_BF16 && d->kv_dtype != CONFU_F32) return CONFU_ERR_ARG;
+    if (d->kv_dtype != CONFU_BF16 && d->kv_dtype != CONFU_F32 && d->kv_dtype != CONFU_FP8_E4M3) return CONFU_ERR_ARG;
+    if (d->kv_dtype == CONFU_FP8_E4M3 && (d->D != 128 || d->Hq / d->Hkv > 4 || d->S > 128)) return CONFU_ERR_UNSUPPORTED;
     if (d->T > CONFU_MAX_TREE || d->C > CONFU_MAX_TREE) return CONFU_ERR_UNSUPPORTED;
     if (!(d->sm_scale >= 0.f)) return CONFU_ERR_ARG;
     return CONFU_OK;
@@ -43,6 +44,14 @@ namespace confu {
 cudaError_t launch_bounded_wait(unsigned long long limit_ns, int32_t* status, cudaStream_t st);
 bool tc_attention_supported(const confu_dims& d);
 bool pair_attention_supported(const confu_dims& d, int sm_count);
+bool fp8_attention_supported(const confu_dims& d);
+cudaError_t launch_attention_fp8(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
+                                 const void* v_cache, int64_t n_slots, const SlotMap& map,
+                                 const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
+                                 void* partials, void* out, float* lse, int32_t* status, cudaStream_t st);
+cudaError_t launch_append_fp8(int B, int R, int Hkv, int D, const void* k_rows, const void* v_rows, void* k_cache,
+                              void* v_cache, const SlotMap& map, const int32_t* prefix_len, const float* k_scale,
+                              const float* v_scale, cudaStream_t st);
 cudaError_t launch_attention_pair(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,
                                   const void* v_cache, int64_t n_slots, const SlotMap& map,
                                   const int32_t* prefix_len, const void* k_soft, const void* v_soft, const void* plan,
@@ -60,6 +69,11 @@ namespace {
 int resolve_attention_path(const confu_ctx* ctx, const confu_dims& d)
 {
     const bool tc = tc_attention_supported(d), pair = pair_attention_supported(d, ctx->sm_count);
+    if (d.kv_dtype == CONFU_FP8_E4M3) {         // one kernel serves E4M3 caches
+        if (!ctx->k_scale) return CONFU_ERR_UNSUPPORTED;
+        const bool ok = ctx->attention_path == CONFU_ATTENTION_AUTO || ctx->attention_path == CONFU_ATTENTION_TENSOR;
+        return ok && fp8_attention_supported(d) ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ERR_UNSUPPORTED;
+    }
     switch (ctx->attention_path) {
         case CONFU_ATTENTION_GENERIC: return CONFU_ATTENTION_GENERIC;
         case CONFU_ATTENTION_TENSOR: return tc ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ERR_UNSUPPORTED;
@@ -92,6 +106,7 @@ int confu_create(confu_ctx** out, int device)
     c->block_table = nullptr;
     c->max_pages = 0;
     c->last_error = cudaSuccess;
+    c->k_scale = c->v_scale = nullptr;
     c->attention_path = CONFU_ATTENTION_AUTO;
     c->wait_ns = 2000000000ull;
     cudaError_t e = cudaSetDevice(device);
@@ -132,6 +147,15 @@ int confu_set_paging(confu_ctx* ctx, const int32_t* block_table, int32_t max_pag
     if (block_table && max_pages <= 0) return CONFU_ERR_ARG;
     ctx->block_table = block_table;
     ctx->max_pages = block_table ? max_pages : 0;
+    return CONFU_OK;
+}
+
+int confu_set_kv_scales(confu_ctx* ctx, const float* k_scale, const float* v_scale)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    if ((k_scale == nullptr) != (v_scale == nullptr)) return CONFU_ERR_ARG;
+    ctx->k_scale = k_scale;
+    ctx->v_scale = v_scale;
     return CONFU_OK;
 }
 
@@ -245,6 +269,9 @@ int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims, const void* q, 
     if (path == CONFU_ATTENTION_TENSOR_PAIR)
         e = launch_attention_pair(ctx, *dims, q, k_cache, v_cache, n_slots, map, prefix_len, k_soft, v_soft,
                                   use_plan, ws + ws_partial_offset(dims), out, lse, status, st);
+    else if (path == CONFU_ATTENTION_TENSOR && dims->kv_dtype == CONFU_FP8_E4M3)
+        e = launch_attention_fp8(ctx, *dims, q, k_cache, v_cache, n_slots, map, prefix_len, k_soft, v_soft,
+                                 use_plan, ws + ws_partial_offset(dims), out, lse, status, st);
     else if (path == CONFU_ATTENTION_TENSOR)
         e = launch_attention_tc(ctx, *dims, q, k_cache, v_cache, n_slots, map, prefix_len, k_soft, v_soft,
                                 use_plan, ws + ws_partial_offset(dims), out, lse, status, st);
@@ -322,7 +349,7 @@ int confu_kv_compact(confu_ctx* ctx, const confu_dims* dims, int32_t n_layers, v
     if (!ctx->block_table && !seq_start) return CONFU_ERR_ARG;
     const SlotMap map = {seq_start, ctx->block_table, ctx->max_pages};
     if (n_layers > 0 && (!k_cache_layers || !v_cache_layers)) return CONFU_ERR_ARG;
-    const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : 4);
+    const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : dims->kv_dtype == CONFU_F32 ? 4 : 1);
     cudaError_t e = launch_compact(ctx, dims->B, dims->T, n_layers, row_bytes, k_cache_layers, v_cache_layers, map,
                                    prefix_len, accept_len, path, new_prefix_len, status, (cudaStream_t)stream);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);
@@ -339,7 +366,13 @@ int confu_kv_append(confu_ctx* ctx, const confu_dims* dims, const void* k_rows, 
     if (!ctx->block_table && !seq_start) return CONFU_ERR_ARG;
     const SlotMap map = {seq_start, ctx->block_table, ctx->max_pages};
     if (misaligned(k_rows) || misaligned(v_rows) || misaligned(k_cache) || misaligned(v_cache)) return CONFU_ERR_ALIGN;
-    const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : 4);
+    const int64_t row_bytes = (int64_t)dims->Hkv * dims->D * (dims->kv_dtype == CONFU_BF16 ? 2 : dims->kv_dtype == CONFU_F32 ? 4 : 1);
+    if (dims->kv_dtype == CONFU_FP8_E4M3) {
+        if (!ctx->k_scale) return CONFU_ERR_UNSUPPORTED;
+        cudaError_t e8 = launch_append_fp8(dims->B, dims->T + dims->C, dims->Hkv, dims->D, k_rows, v_rows, k_cache, v_cache,
+                                           map, prefix_len, ctx->k_scale, ctx->v_scale, (cudaStream_t)stream);
+        return e8 == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e8);
+    }
     cudaError_t e = launch_append(dims->B, dims->T + dims->C, row_bytes, k_rows, v_rows, k_cache, v_cache, map,
                                   prefix_len, (cudaStream_t)stream);
     return e == cudaSuccess ? CONFU_OK : cuda_fail(ctx, e);

@@ -515,6 +515,7 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
     prm.G = G;
     prm.c = (d.sm_scale != 0.f ? d.sm_scale : 1.f / sqrtf((float)d.D)) * 1.4426950408889634f;
     prm.wait_ns = ctx->wait_ns;
+    prm.k_scale = prm.v_scale = nullptr;
     const size_t smem = sizeof(SharedStorage) + 1024;
     static OncePerDevice attr_done;
     {

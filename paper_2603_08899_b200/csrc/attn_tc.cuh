@@ -23,6 +23,8 @@ struct Params {
     int G;
     float c;             // sm_scale * log2(e)
     unsigned long long wait_ns;   // limit of every wait on an mbarrier (wall clock)
+    const float* k_scale;         // E4M3 cache: value = code * scale[kv head] (device, [Hkv]); unused otherwise
+    const float* v_scale;
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)

@@ -121,6 +121,8 @@ struct Ctx {
     const int32_t* block_table;    // paged pools when set (confu_set_paging)
     int32_t max_pages;
     cudaError_t last_error;
+    const float* k_scale;          // E4M3 caches: per-kv-head scales (confu_set_kv_scales)
+    const float* v_scale;
     int attention_path;            // CONFU_ATTENTION_* (confu_set_option)
     unsigned long long wait_ns;    // limit of the bounded waits inside the kernels
 };

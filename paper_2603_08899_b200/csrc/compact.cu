@@ -73,6 +73,50 @@ __global__ void __launch_bounds__(128) append_kernel(int R, int64_t row_vecs, co
     for (int64_t c = threadIdx.x; c < row_vecs; c += blockDim.x) dst[c] = src[c];
 }
 
+// E4M3 cache: cache[...][g][d] = e4m3(rows[b][r][g][d] / scale[g]) (quotient in fp32, round to nearest even,
+// saturating at 448).  One thread per 16 output bytes.
+__global__ void __launch_bounds__(128) append_fp8_kernel(int R, int Hkv, int D, const __nv_bfloat16* __restrict__ k_rows,
+                                                         const __nv_bfloat16* __restrict__ v_rows, uint8_t* __restrict__ k_cache,
+                                                         uint8_t* __restrict__ v_cache, const SlotMap map,
+                                                         const int32_t* __restrict__ prefix_len,
+                                                         const float* __restrict__ k_scale, const float* __restrict__ v_scale)
+{
+    const int r = blockIdx.x, b = blockIdx.y, kv = blockIdx.z;
+    const int row_elems = Hkv * D;
+    const __nv_bfloat16* src = (kv ? v_rows : k_rows) + ((size_t)b * R + r) * row_elems;
+    uint8_t* dst = (kv ? v_cache : k_cache) + (size_t)pool_slot(map, b, (int64_t)prefix_len[b] + r) * row_elems;
+    const float* scale = kv ? v_scale : k_scale;
+    for (int i = threadIdx.x * 16; i < row_elems; i += blockDim.x * 16) {
+        const float s = scale[i / D];
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float x[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) x[j] = __bfloat162float(src[i + 4 * q + j]) / s;
+            uint32_t word;
+            asm("{\n\t.reg .b16 lo, hi;\n\t"
+                "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+                "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+                "mov.b32 %0, {lo, hi};\n\t}"
+                : "=r"(word)
+                : "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]));
+            w[q] = word;
+        }
+        *reinterpret_cast<uint4*>(dst + i) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+cudaError_t launch_append_fp8(int B, int R, int Hkv, int D, const void* k_rows, const void* v_rows, void* k_cache,
+                              void* v_cache, const SlotMap& map, const int32_t* prefix_len, const float* k_scale,
+                              const float* v_scale, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    append_fp8_kernel<<<dim3(R, B, 2), 128, 0, st>>>(R, Hkv, D, (const __nv_bfloat16*)k_rows, (const __nv_bfloat16*)v_rows,
+                                                     (uint8_t*)k_cache, (uint8_t*)v_cache, map, prefix_len, k_scale, v_scale);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_append(int B, int R, int64_t row_bytes, const void* k_rows, const void* v_rows, void* k_cache,
                           void* v_cache, const SlotMap& map, const int32_t* prefix_len, cudaStream_t st)
 {
