@@ -33,11 +33,12 @@ UNIT = "steps/s"
 def attention_bytes_per_layer(cfg, plen):
     """Algorithmic HBM bytes of one attention launch: every K and V row of every sequence read once
     (prefix + the R rows' own slots), the soft-prompt K/V once, Q read and O written once."""
-    es = 2 if cfg.kv_dtype == torch.bfloat16 else 4
+    es = {torch.bfloat16: 2, torch.float32: 4, torch.float8_e4m3fn: 1}[cfg.kv_dtype]      # cache entries
+    qs = 2 if cfg.kv_dtype == torch.float8_e4m3fn else es                                   # q and out (bf16 over an E4M3 cache)
     row = cfg.Hkv * cfg.D * es
     kv = 2 * row * int((plen.to(torch.int64) + cfg.R).sum())
     soft = 2 * row * cfg.S
-    qo = 2 * cfg.B * cfg.R * cfg.Hq * cfg.D * es
+    qo = 2 * cfg.B * cfg.R * cfg.Hq * cfg.D * qs
     return kv + soft + qo
 
 
@@ -49,7 +50,7 @@ def attention_flops_per_layer(cfg, plen):
 def step_bytes(cfg, plen, accept_len_mean):
     es = 2 if cfg.logit_dtype == torch.bfloat16 else 4
     logits = 2 * cfg.B * cfg.T * cfg.V * es
-    row = cfg.Hkv * cfg.D * (2 if cfg.kv_dtype == torch.bfloat16 else 4)
+    row = cfg.Hkv * cfg.D * {torch.bfloat16: 2, torch.float32: 4, torch.float8_e4m3fn: 1}[cfg.kv_dtype]
     compact = int(2 * 2 * accept_len_mean * row * cfg.L * cfg.B)
     return cfg.L * attention_bytes_per_layer(cfg, plen) + logits + compact
 
@@ -67,7 +68,9 @@ def attention_lens(cfg, plen, launch_s, clocks, peaks, sm_count):
     peaks (the larger of bytes / copy bandwidth and FLOPs / sustained bf16 matmul rate)."""
     a_bytes = attention_bytes_per_layer(cfg, plen)
     a_flops = attention_flops_per_layer(cfg, plen)
-    t_hbm, t_tc = a_bytes / (peaks["hbm_gbs"] * 1e9), a_flops / (peaks["bf16_tflops"] * 1e12)
+    # tensor ceiling of the type the products run in: E4M3 products at twice the measured bf16 rate (nominal ratio)
+    tc_peak = peaks["bf16_tflops"] * (2.0 if cfg.kv_dtype == torch.float8_e4m3fn else 1.0)
+    t_hbm, t_tc = a_bytes / (peaks["hbm_gbs"] * 1e9), a_flops / (tc_peak * 1e12)
     gbs, tf = a_bytes / launch_s / 1e9, a_flops / launch_s / 1e12
     mhz = clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None
     tiles = key_tiles_per_layer(cfg, plen)
@@ -75,7 +78,7 @@ def attention_lens(cfg, plen, launch_s, clocks, peaks, sm_count):
             "floor_us": {"hbm": t_hbm * 1e6, "tensor": t_tc * 1e6},
             "bytes_per_launch": a_bytes, "flops_per_launch": a_flops, "key_tiles_per_launch": tiles,
             "hbm_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0,
-            "tensor_tflops": tf, "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops"],
+            "tensor_tflops": tf, "tensor_peak_tflops": tc_peak, "frac_of_measured_bf16_sustained": tf / tc_peak,
             # clock-independent figures: time x median SM clock under load
             "mcycles_per_launch": None if mhz is None else launch_s * mhz,
             "cycles_per_key_tile_per_sm": None if mhz is None else launch_s * mhz * 1e6 * sm_count / max(tiles, 1)}
@@ -90,7 +93,8 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
 
 
-KERNEL_SOURCES = {"attention_pair_kernel": ("attn_tc2.cu", "tc_walk.cuh", "tc_ptx.cuh", "attn_tc.cuh"),
+KERNEL_SOURCES = {"attention_fp8_kernel": ("attn_fp8.cu", "tc_walk.cuh", "tc_ptx.cuh", "attn_tc.cuh"),
+                  "attention_pair_kernel": ("attn_tc2.cu", "tc_walk.cuh", "tc_ptx.cuh", "attn_tc.cuh"),
                   "attention_tc_kernel": ("attn_tc.cu", "tc_walk.cuh", "tc_ptx.cuh", "attn_tc.cuh"),
                   "attention_generic_kernel": ("attn_generic.cu",)}
 
@@ -271,11 +275,13 @@ def build_workload(cfg, device, rank, temperature=1.0):
     parent, owner = inputs.trees(cfg)
     plen = inputs.prefix_lens(cfg)
     seq_start, n_slots = inputs.cache_layout(cfg, plen)
-    q, k, v, ks, vs, out = [], [], [], [], [], []
+    q, k, v, ks, vs, out, scales = [], [], [], [], [], [], []
     for l in range(cfg.L):
         t = inputs.layer_tensors(cfg, l, n_slots, device=device)
         q.append(t["q"]); k.append(t["k_cache"]); v.append(t["v_cache"]); ks.append(t["k_soft"]); vs.append(t["v_soft"])
         out.append(torch.empty_like(t["q"]))
+        if "k_scale" in t:
+            scales.append((t["k_scale"], t["v_scale"]))
     tl, dl = inputs.logits(cfg, device=device)
     tok = inputs.draft_tokens(cfg, parent, dl, temperature)
     u = inputs.uniforms(cfg)
@@ -284,7 +290,8 @@ def build_workload(cfg, device, rank, temperature=1.0):
         from paper_2603_08899_b200 import binding as cb
         cb.confu_set_option(step.ctx, cb.OPT_ATTENTION_PATH, ATTENTION_PATH)
     step.bind(q, k, v, ks if cfg.S else None, vs if cfg.S else None, out, seq_start.to(device), plen.to(device),
-              parent.to(device), owner.to(device) if cfg.C else None, tl, dl, tok.to(device), u.to(device))
+              parent.to(device), owner.to(device) if cfg.C else None, tl, dl, tok.to(device), u.to(device),
+              kv_scales=scales or None)
     host = {"parent": parent, "owner": owner, "plen": plen, "seq_start": seq_start, "tok": tok, "u": u}
     return cfg, step, host
 
@@ -568,7 +575,8 @@ def run_ours(args, cfg):
             setattr(step, name, None)
         torch.cuda.empty_cache()
         others = {}
-        for name, temperature in (("llama3b", 1.0), ("llama8b", 1.0), ("qwen4b", 1.0), ("qwen4b", 0.0), ("batch32_2t", 1.0)):
+        for name, temperature in (("llama3b", 1.0), ("llama8b", 1.0), ("qwen4b", 1.0), ("qwen4b", 0.0), ("batch32_2t", 1.0),
+                                  ("batch32_fp8", 1.0)):
             key = name if temperature > 0 else name + "_greedy"
             others[key] = time_other_workload(name, temperature, device, local, peaks)
     else:

@@ -70,7 +70,6 @@ int resolve_attention_path(const confu_ctx* ctx, const confu_dims& d)
 {
     const bool tc = tc_attention_supported(d), pair = pair_attention_supported(d, ctx->sm_count);
     if (d.kv_dtype == CONFU_FP8_E4M3) {         // one kernel serves E4M3 caches
-        if (!ctx->k_scale) return CONFU_ERR_UNSUPPORTED;
         const bool ok = ctx->attention_path == CONFU_ATTENTION_AUTO || ctx->attention_path == CONFU_ATTENTION_TENSOR;
         return ok && fp8_attention_supported(d) ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ERR_UNSUPPORTED;
     }
@@ -255,6 +254,7 @@ int confu_tree_attention(confu_ctx* ctx, const confu_dims* dims, const void* q, 
     if (!ctx->workspace || ctx->workspace_bytes < ws_total(ctx, dims)) return CONFU_ERR_WORKSPACE;
     const int path = resolve_attention_path(ctx, *dims);
     if (path < 0) return path;
+    if (dims->kv_dtype == CONFU_FP8_E4M3 && !ctx->k_scale) return CONFU_ERR_UNSUPPORTED;      // an E4M3 cache means nothing without its scales
     cudaStream_t st = (cudaStream_t)stream;
     char* ws = (char*)ctx->workspace;
     const void* use_plan = plan;

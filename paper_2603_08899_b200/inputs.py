@@ -76,6 +76,11 @@ CONFIGS = {
                                prefix=4096, tree="random", kv_dtype=torch.bfloat16,
                                logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",
                                temperatures=(1.0,), seed=8),
+    # the batched workload over an 8-bit floating point (E4M3) cache with one scale per KV head
+    "batch32_fp8": VerifyConfig("batch32_fp8", B=32, L=32, Hq=32, Hkv=8, D=128, T=60, C=4, S=16, V=128256,
+                                prefix=(512, 16384), tree="random", kv_dtype=torch.float8_e4m3fn,
+                                logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",
+                                temperatures=(1.0,), seed=5),
     "batch32_2t": VerifyConfig("batch32_2t", B=32, L=32, Hq=32, Hkv=8, D=128, T=60, C=60, S=16, V=128256,
                                prefix=(512, 16384), tree="random", kv_dtype=torch.bfloat16,
                                logit_dtype=torch.bfloat16, sigma_logit=3.0, draft="noise",
@@ -188,12 +193,22 @@ def layer_tensors(cfg: VerifyConfig, layer: int, n_slots: int, device="cpu", tre
     tree_key_gain > 1 scales the keys of the tree slots so that tree columns dominate the softmax
     (makes mask mistakes visible at long prefixes)."""
     g = _gen(cfg, 100 + layer, device)
-    dt = cfg.kv_dtype
+    fp8 = cfg.kv_dtype == torch.float8_e4m3fn
+    dt = torch.bfloat16 if fp8 else cfg.kv_dtype
     q = _randn((cfg.B, cfg.R, cfg.Hq, cfg.D), g, device, dt)
     k = _randn((n_slots, cfg.Hkv, cfg.D), g, device, dt)
     v = _randn((n_slots, cfg.Hkv, cfg.D), g, device, dt)
     ks = _randn((cfg.S, cfg.Hkv, cfg.D), g, device, dt) if cfg.S else None
     vs = _randn((cfg.S, cfg.Hkv, cfg.D), g, device, dt) if cfg.S else None
+    if fp8:
+        # E4M3 cache entries (bytes) with one scale per KV head; q stays bf16.  (The library's cast is
+        # input preparation here: the synthetic cache just has to hold valid codes.)
+        k_scale, v_scale = fp8_scales(cfg, layer)
+        to8 = lambda x, s: (x.float() / s.to(x.device).view(1, -1, 1)).clamp(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+        out = {"q": q, "k_cache": to8(k, k_scale), "v_cache": to8(v, v_scale),
+               "k_soft": to8(ks, k_scale) if cfg.S else None, "v_soft": to8(vs, v_scale) if cfg.S else None,
+               "k_scale": k_scale.to(device), "v_scale": v_scale.to(device)}
+        return out
     if tree_key_gain != 1.0:
         for b in range(cfg.B):
             lo = int(seq_start[b]) + int(prefix_len[b])

@@ -35,8 +35,10 @@ class VerifyStep:
             self.own_ctx = False
 
     def bind(self, q_layers, k_layers, v_layers, k_soft, v_soft, out_layers, seq_start, prefix_len, parent,
-             con_owner, target_logits, draft_logits, tokens, uniforms):
-        """Remember the (device) tensors of a step; lists have one entry per layer."""
+             con_owner, target_logits, draft_logits, tokens, uniforms, kv_scales=None):
+        """Remember the (device) tensors of a step; lists have one entry per layer.  kv_scales: for an
+        E4M3 cache, one (k_scale, v_scale) pair of fp32 [Hkv] tensors per layer."""
+        self.kv_scales = kv_scales
         self.q, self.k, self.v, self.ks, self.vs, self.out = q_layers, k_layers, v_layers, k_soft, v_soft, out_layers
         self.seq_start, self.prefix_len, self.parent, self.con_owner = seq_start, prefix_len, parent, con_owner
         self.tl, self.dl, self.tokens, self.uniforms = target_logits, draft_logits, tokens, uniforms
@@ -48,6 +50,8 @@ class VerifyStep:
         cb.confu_tree_plan(self.ctx, self.dims, self.seq_start, self.prefix_len, self.parent, self.con_owner,
                            self.plan, self.status)
         for l in range(len(self.q)):
+            if self.kv_scales is not None:
+                cb.confu_set_kv_scales(self.ctx, *self.kv_scales[l])
             cb.confu_tree_attention(self.ctx, self.dims, self.q[l], self.k[l], self.v[l], self.n_slots,
                                     self.seq_start, self.prefix_len,
                                     self.ks[l] if self.ks is not None else None,
@@ -62,6 +66,8 @@ class VerifyStep:
     def run_layers(self):
         """The L attention calls with the plan built by run_plan()."""
         for l in range(len(self.q)):
+            if self.kv_scales is not None:
+                cb.confu_set_kv_scales(self.ctx, *self.kv_scales[l])
             cb.confu_tree_attention(self.ctx, self.dims, self.q[l], self.k[l], self.v[l], self.n_slots,
                                     self.seq_start, self.prefix_len,
                                     self.ks[l] if self.ks is not None else None,
@@ -120,14 +126,16 @@ def sm_count(step):
 
 
 def uses_tensor_core_path(cfg):
-    """Mirror of the library's dispatch rule: bf16, head dim 128, at most 4 query heads per KV head."""
-    return cfg.kv_dtype == torch.bfloat16 and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
+    """Mirror of the library's dispatch rule: bf16 or E4M3 cache, head dim 128, at most 4 query heads per KV head."""
+    return cfg.kv_dtype in (torch.bfloat16, torch.float8_e4m3fn) and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
 
 
 def attention_kernel_name(cfg):
     """Mirror of the library's choice of attention kernel (CONFU_ATTENTION_AUTO)."""
     if not uses_tensor_core_path(cfg):
         return "attention_generic_kernel"
+    if cfg.kv_dtype == torch.float8_e4m3fn:
+        return "attention_fp8_kernel"
     n_rg = (cfg.T + cfg.C + 63) // 64
     sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count if torch.cuda.is_available() else 148
     few_pairs = cfg.B * cfg.Hkv * n_rg <= sms // 2
