@@ -560,8 +560,9 @@ static bool make_byte_map(CUtensorMap* map, const void* base, uint64_t rows, uin
     const cuuint64_t strides[2] = {(cuuint64_t)kD, heads * kD};
     const cuuint32_t box[3] = {(cuuint32_t)kD, 1, (cuuint32_t)kTileKeys};
     const cuuint32_t estr[3] = {1, 1, 1};
+    // (rows of one head are 128 B apart from the next head's: promoting L2 fetches to 256 B would read the neighbour too)
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
