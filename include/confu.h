@@ -115,7 +115,9 @@ int confu_set_workspace(confu_ctx* ctx, void* device_ptr, size_t bytes);
  * in page block_table[b][s / 128] at offset s % 128, i.e. at pool slot 128 * page + s % 128.
  * block_table: DEVICE int32 [B][max_pages], with at least ceil((prefix_len[b] + R) / 128) valid
  * page ids per sequence; read by every later call until it is cleared (NULL); seq_start is then
- * ignored and may be NULL, and n_slots must be a whole number of pages.  The paper has no cache
+ * ignored and may be NULL, and n_slots must be a whole number of pages.  Page ids are the caller's: an id
+ * past the pool reads as zeros in confu_tree_attention (the tile loads are bounds-checked by the hardware) but is an
+ * out-of-bounds store in confu_kv_append and confu_kv_compact, which do not know the pool's size.  The paper has no cache
  * layout (Sec. 3.1 only says the K/V of accepted tokens are kept); pages of one key tile are what
  * serving engines use.
  */

@@ -9,9 +9,10 @@
 //     scale of its own (largest magnitude -> 448) and writes it into the Q tile the tensor pipe reads;
 //     the row's scale, the cache's per-head K scale and the softmax scale are one factor of the
 //     exponent's argument;
-//   - P is handed over as E4M3 too, shifted by 2^7 so that the weights use the format's range (the
-//     reference maximum moves whenever the running maximum grows by more than 1, which keeps every
-//     weight under 2^8.x <= 448); numerator and denominator carry the same shift;
+//   - P is handed over as E4M3 too, shifted by 2^5 so that the weights use the format's range (the
+//     reference maximum moves whenever the running maximum grows by more than 3, which keeps every
+//     weight at or under 2^8 < 448, while weights down to 2^-14 of the reference survive; moving it
+//     more eagerly costs a rescale of O each time); numerator and denominator carry the same shift;
 //   - the per-head V scale multiplies the output rows (or the partial results) at the end of a run.
 #include "tc_walk.cuh"
 
@@ -23,10 +24,10 @@ namespace f8 {
 constexpr int kThreads = 384;            // warps 0-3: softmax of M tile 0, 4-7: of M tile 1, 8: TMA, 9: MMA, 10: ragged tail of V
 constexpr int kStages = 3;               // ring of stages; stage g = [V of the CTA's g-1st key tile | K of its g-th]
 constexpr int kTile8 = kTileKeys * kD;   // a 128-key tile of E4M3 bytes: 16 KB, rows of 128 B
-constexpr float kPShift = 7.f;           // weights are handed over as 2^(x - m + 7)
+constexpr float kPShift = 5.f;           // weights are handed over as 2^(x - m + 5)
 constexpr int kQBytes = 2 * kTileBytes;             // two M tiles
 constexpr uint32_t kTmemCols = 512;                 // S0 | S1 | O0 | O1, 128 columns each; P_t overlays S_t
-constexpr float kRescaleThreshold = 1.f;            // the reference maximum follows the running maximum within 2^1 (E4M3 range)
+constexpr float kRescaleThreshold = 3.f;            // the reference maximum follows the running maximum within 2^3: weights stay <= 2^8 < 448
 
 struct SharedStorage {
     alignas(1024) uint8_t q[kQBytes];                    // Q as it arrives: bf16, two M tiles x two 64-wide halves
@@ -401,7 +402,7 @@ __device__ void softmax_role(SharedStorage& sh, const Params& prm, const PlanVie
         float4* xp = sh.xpose[threadIdx.x >> 5];
         const bool whole = s.part_slot < 0;
         // O holds sum of weight * V code: the head's V scale turns codes into values; a partial result keeps
-        // its sum of weights apart (both carry the 2^7 shift of the weights)
+        // its sum of weights apart (both carry the shift of the weights)
         const float v_scale = __ldg(prm.v_scale + s.g);
         const float inv_l = whole ? v_scale / l : v_scale;
         // where this lane's pieces go: row 8 kk + lane / 4 of the warp's 32 (output), row 4 kk + lane / 8 (partial)
