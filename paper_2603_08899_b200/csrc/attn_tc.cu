@@ -381,9 +381,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
 {
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& sh = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // the kernels before this one have completed
-    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
-    if ((int)blockIdx.x >= pv.hdr->n_ctas) return;
     const int warp = threadIdx.x >> 5;
 
     if (threadIdx.x == 0) {
@@ -411,8 +408,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
+    // Everything above touches only this kernel's own shared and tensor memory, so it runs while the
+    // kernel before this one in the stream drains.  From here on global memory is read and written:
+    // every CTA waits until the kernels before this one have completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
 
-    if (warp < 8) {
+    if ((int)blockIdx.x >= pv.hdr->n_ctas) {
+        // nothing to do: straight to the teardown, which releases tensor memory
+    } else if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         const int t = warp >> 2;
         if (t < prm.n_mt) softmax_role(sh, prm, pv, tmem, t);
@@ -525,8 +529,9 @@ cudaError_t launch_attention_tc(const Ctx* ctx, const confu_dims& d, const void*
         if (e != cudaSuccess) return e;
     }
     // Launched as a programmatic dependent of whatever precedes it in the stream: its CTAs may be
-    // scheduled while the predecessor drains; the kernel waits (griddepcontrol.wait, first thing) for
-    // the predecessor's completion and memory flush before it touches global memory.
+    // scheduled while the predecessor drains; the kernel sets up its barriers and tensor memory, then
+    // waits (griddepcontrol.wait) for the predecessor's completion and memory flush before it touches
+    // global memory.
     cudaLaunchAttribute pdl[1];
     pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl[0].val.programmaticStreamSerializationAllowed = 1;

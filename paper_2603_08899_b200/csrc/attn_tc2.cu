@@ -546,15 +546,9 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
 {
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& sh = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // the kernels before this one have completed
-    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
-    // (both CTAs of a pair take the same way out of the next two tests)
-    if ((int)(blockIdx.x >> 1) >= pv.hdr->n_ctas) return;
-    if (pv.hdr->paired != 1) {                              // the plan lists runs per CTA, not per CTA pair
-        if (blockIdx.x == 0 && prm.status)
-            for (int b = threadIdx.x; b < prm.d.B; b += kThreads) prm.status[b] = CONFU_ST_BAD_PLAN;
-        return;
-    }
+    // The kernel after this one in the stream may be scheduled as soon as every CTA has got here; it
+    // waits for this grid's completion itself before it touches anything this grid reads or writes.
+
     const int warp = threadIdx.x >> 5;
     const uint32_t rank = cluster_ctarank();
 
@@ -593,8 +587,20 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
     cluster_sync_all();                                     // the other CTA's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem = sh.tmem_base;
+    // Everything above touches only this kernel's own shared and tensor memory, so it runs while the
+    // kernel before this one in the stream drains.  From here on global memory is read and written:
+    // every CTA waits until the kernels before this one have completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
+    // (both CTAs of a pair take the same way through the next two tests)
+    const bool listed = (int)(blockIdx.x >> 1) < pv.hdr->n_ctas;
+    const bool pair_plan = pv.hdr->paired == 1;             // the plan lists runs per CTA pair, not per CTA
+    if (!pair_plan && blockIdx.x == 0 && prm.status)
+        for (int b = threadIdx.x; b < prm.d.B; b += kThreads) prm.status[b] = CONFU_ST_BAD_PLAN;
 
-    if (warp < 8) {
+    if (!listed || !pair_plan) {
+        // nothing to do: straight to the teardown, which releases tensor memory
+    } else if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         softmax_role(sh, prm, pv, tmem, rank);
     } else if (warp == 8) {

@@ -23,6 +23,7 @@ __device__ __forceinline__ void zero_row(const Params& prm, int b, int g, int r,
 // 256-byte lines.
 __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
 {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the attention kernel has completed
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
     const int pair = blockIdx.x, t = blockIdx.y;
@@ -81,6 +82,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
 constexpr int kCombineRowsPerBlock = 16;
 __global__ void __launch_bounds__(32 * kCombineRowsPerBlock) combine_wide_kernel(const Params prm)
 {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the attention kernel has completed
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
     const int pair = blockIdx.x, t = blockIdx.y;
