@@ -68,10 +68,11 @@ namespace {
 // (never _AUTO), or a negative error code when a forced path cannot take them.
 int resolve_attention_path(const confu_ctx* ctx, const confu_dims& d)
 {
-    const bool tc = tc_attention_supported(d), pair = pair_attention_supported(d, ctx->sm_count);
+    // (a share of the work is walked by one CTA, or CTA pair, per group of 64 query rows: at least two of them)
+    const bool tc = tc_attention_supported(d) && ctx->sm_count >= 2, pair = pair_attention_supported(d, ctx->sm_count);
     if (d.kv_dtype == CONFU_FP8_E4M3) {         // one kernel serves E4M3 caches
         const bool ok = ctx->attention_path == CONFU_ATTENTION_AUTO || ctx->attention_path == CONFU_ATTENTION_TENSOR;
-        return ok && fp8_attention_supported(d) ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ERR_UNSUPPORTED;
+        return ok && fp8_attention_supported(d) && ctx->sm_count >= 2 ? (int)CONFU_ATTENTION_TENSOR : (int)CONFU_ERR_UNSUPPORTED;
     }
     switch (ctx->attention_path) {
         case CONFU_ATTENTION_GENERIC: return CONFU_ATTENTION_GENERIC;

@@ -644,7 +644,7 @@ bool make_tile_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t h
 bool pair_attention_supported(const confu_dims& d, int sm_count)
 {
     const int G = d.Hq / d.Hkv;
-    return d.kv_dtype == CONFU_BF16 && d.D == 128 && G <= 4 && d.S <= 128 && d.T + d.C > 32 && sm_count >= 2;
+    return d.kv_dtype == CONFU_BF16 && d.D == 128 && G <= 4 && d.S <= 128 && d.T + d.C > 32 && sm_count >= 4;
 }
 
 cudaError_t launch_attention_pair(const Ctx* ctx, const confu_dims& d, const void* q, const void* k_cache,

@@ -39,10 +39,11 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
             zero_row(prm, b, g, kGroupRows * rg + 32 * t + lane_row / G, lane_row % G, lane);
         return;
     }
-    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
-    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
-    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
-    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
+    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas / prm.n_rg;
+    // key tile q of (sequence, kv head) sits at position F + q of the cost line; position x belongs to lane
+    // floor(((x + 1) * n - 1) / N) of the n lanes, and row group rg of lane c is walked by CTA c * n_rg + rg
+    const int64_t F = pv.tile_base[b] + (int64_t)g * (nt + kPairOverheadTiles) + kPairOverheadTiles;
+    const int c_first = (int)(((F + 1) * n - 1) / N) * prm.n_rg + rg, c_last = (int)(((F + nt) * n - 1) / N) * prm.n_rg + rg;
     if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
     const size_t slot_floats = partial_slot_bytes() / sizeof(float);
     for (int lane_row = blockIdx.z * 32 + warp; lane_row < min(32 * G, (int)blockIdx.z * 32 + 32); lane_row += 8) {
@@ -50,13 +51,13 @@ __global__ void __launch_bounds__(256) combine_kernel(const Params prm)
         if (r >= R) break;
         const int row = t * 128 + lane_row;
         float M = -INFINITY;
-        for (int cta = c_first; cta <= c_last; ++cta) {
+        for (int cta = c_first; cta <= c_last; cta += prm.n_rg) {
             const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
             M = fmaxf(M, slot[(size_t)kPartRows * kPartD + row]);
         }
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         float L = 0.f;
-        for (int cta = c_first; cta <= c_last; ++cta) {
+        for (int cta = c_first; cta <= c_last; cta += prm.n_rg) {
             const float* slot = prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
             const float m = slot[(size_t)kPartRows * kPartD + row];
             const float w = (m == -INFINITY) ? 0.f : ex2(m - M);
@@ -100,16 +101,17 @@ __global__ void __launch_bounds__(32 * kCombineRowsPerBlock) combine_wide_kernel
         zero_row(prm, b, g, r, hl, lane);
         return;
     }
-    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas;
-    // key tile q of the pair sits at position F + q of the cost line; position x belongs to CTA floor(((x + 1) * n - 1) / N)
-    const int64_t F = pv.tile_base[b] + (int64_t)(pair % per_seq) * (nt + kPairOverheadTiles) + kPairOverheadTiles;
-    const int c_first = (int)(((F + 1) * n - 1) / N), c_last = (int)(((F + nt) * n - 1) / N);
+    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas / prm.n_rg;
+    // key tile q of (sequence, kv head) sits at position F + q of the cost line; position x belongs to lane
+    // floor(((x + 1) * n - 1) / N) of the n lanes, and row group rg of lane c is walked by CTA c * n_rg + rg
+    const int64_t F = pv.tile_base[b] + (int64_t)g * (nt + kPairOverheadTiles) + kPairOverheadTiles;
+    const int c_first = (int)(((F + 1) * n - 1) / N) * prm.n_rg + rg, c_last = (int)(((F + nt) * n - 1) / N) * prm.n_rg + rg;
     if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
     const int row = t * 128 + lane_row;
-    const int n_parts = c_last - c_first + 1;
+    const int n_parts = (c_last - c_first) / prm.n_rg + 1;
     const size_t slot_floats = partial_slot_bytes() / sizeof(float);
-    auto slot_of = [&](int p) {                         // part p of the pair: the partial slot of CTA c_first + p
-        const int cta = c_first + p;
+    auto slot_of = [&](int p) {                         // part p of the pair: the partial slot of the p-th CTA that walked it
+        const int cta = c_first + p * prm.n_rg;
         return prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
     };
     float M = -INFINITY;

@@ -23,15 +23,18 @@ constexpr int kTileKeys = 128;                  // keys per attention tile (tens
 //                             row also sees its own slot and no other contemplate row's: not stored.)
 //   int32  bad[B]             non-zero: malformed tree, sequence skipped
 //   int32  tiles[B]           key tiles of one (sequence, kv head) pair, soft-prompt tile included
-//   int64  tile_base[B + 1]   position of sequence b's first pair on the flat cost line (exclusive scan)
+//   int64  tile_base[B + 1]   position of sequence b's first (sequence, kv head) stretch on the flat cost line (exclusive scan)
 //   int32  seg_begin[kPlanMaxCtas + 1]   CTA c of the tensor-core kernel walks segs[seg_begin[c] .. seg_begin[c+1])
 //   SegDesc segs[B * Hkv * 2 + kPlanMaxCtas]   the runs of key tiles, one pair at a time, of every CTA in walking order
 //
 // The split-KV work is balanced on a "cost line": every (sequence, kv head) pair takes
 // tiles + kPairOverheadTiles consecutive positions (the overhead stands for loading Q, draining
-// the pipeline and writing the output once per pair), pairs in (sequence, head) order.  CTA c of n
-// gets positions [c*N/n, (c+1)*N/n); position q of a pair means key tile q - kPairOverheadTiles,
-// so a CTA whose share ends inside a pair's overhead zone takes none of its tiles.
+// the pipeline and writing the output once per pair), pairs in (sequence, head) order.  The line is
+// cut into n equal shares; share c covers positions [c*N/n, (c+1)*N/n); position q of a pair means
+// key tile q - kPairOverheadTiles, so a share that ends inside a pair's overhead zone takes none of
+// its tiles.  With n_rg groups of 64 query rows (n_rg = 1 or 2) there are n = n_ctas / n_rg shares and
+// CTA c * n_rg + rg walks share c for row group rg: the CTAs of a share read the same K/V tiles at
+// about the same time, so that only the first read of a tile goes to DRAM.
 // ---------------------------------------------------------------------------
 constexpr int kPairOverheadTiles = 4;
 struct PlanHeader {

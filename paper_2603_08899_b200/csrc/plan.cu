@@ -69,15 +69,20 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int units, int 
         int64_t acc = 0;
         for (int b = 0; b < B; ++b) {
             pv.tile_base[b] = acc;
-            // one pair per (kv head, group of 64 query rows)
-            if (pv.tiles[b] > 0) acc += (int64_t)(pv.tiles[b] + kPairOverheadTiles) * d.Hkv * ((R + kGroupRows - 1) / kGroupRows);
+            // one stretch of the line per (sequence, kv head); its groups of 64 query rows are walked side by side
+            if (pv.tiles[b] > 0) acc += (int64_t)(pv.tiles[b] + kPairOverheadTiles) * d.Hkv;
         }
         pv.tile_base[B] = acc;
         PlanHeader h;
         h.B = B; h.Hkv = d.Hkv; h.T = T; h.C = C; h.S = d.S; h.R = R;
         h.n_tiles = acc;
-        h.n_ctas = (int)(acc < (int64_t)units ? acc : (int64_t)units);
-        if (h.n_ctas > kPlanMaxCtas) h.n_ctas = kPlanMaxCtas;
+        // The line is cut into `lanes` shares; CTA lane * n_rg + rg walks the lane's share for row group rg,
+        // so the CTAs of a lane read the same K/V tiles at about the same time (the second read hits L2).
+        const int n_rg0 = (R + kGroupRows - 1) / kGroupRows;
+        int cap = units < kPlanMaxCtas ? units : kPlanMaxCtas;
+        int lanes = cap / n_rg0;
+        if ((int64_t)lanes > acc) lanes = (int)acc;
+        h.n_ctas = lanes * n_rg0;
         h.paired = paired;
         *pv.hdr = h;
     }
@@ -87,12 +92,13 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int units, int 
     // line, first to count its runs, then (behind a prefix sum) to write them down.
     const int n_rg = (R + kGroupRows - 1) / kGroupRows;
     const int64_t N = pv.hdr->n_tiles;
-    const int n_ctas = pv.hdr->n_ctas;
+    const int n_ctas = pv.hdr->n_ctas, n_lanes = n_ctas / n_rg;
     for (int pass = 0; pass < 2; ++pass) {
         const int c = threadIdx.x;
         if (c < n_ctas) {
-            int64_t f = (int64_t)c * N / n_ctas;
-            const int64_t f1 = (int64_t)(c + 1) * N / n_ctas;
+            const int lane = c / n_rg, rg = c % n_rg;
+            int64_t f = (int64_t)lane * N / n_lanes;
+            const int64_t f1 = (int64_t)(lane + 1) * N / n_lanes;
             int n = 0;
             SegDesc* out = pv.segs + (pass ? s_count[c] : 0);
             int lo = 0;
@@ -109,10 +115,9 @@ __global__ void __launch_bounds__(256) plan_kernel(confu_dims d, int units, int 
                 const int t1 = pos + take > kPairOverheadTiles ? pos + take - kPairOverheadTiles : 0;
                 if (t1 <= t0) continue;                    // the share ended inside this pair's overhead zone
                 if (pass) {
-                    const int pair = (int)(local / cost);       // pairs of a sequence: kv head major, row group minor
                     SegDesc d;
                     d.b = lo;
-                    d.g_rg = (pair / n_rg) | ((pair % n_rg) << 16);
+                    d.g_rg = (int)(local / cost) | (rg << 16);       // the stretches of a sequence are in kv-head order
                     d.t0 = t0;
                     d.t1 = t1;
                     d.nt = nt;
