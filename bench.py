@@ -575,9 +575,9 @@ def run_ours(args, cfg):
             setattr(step, name, None)
         torch.cuda.empty_cache()
         others = {}
-        for name, temperature in (("llama3b", 1.0), ("llama8b", 1.0), ("qwen4b", 1.0), ("qwen4b", 0.0), ("batch32_2t", 1.0),
-                                  ("batch32_fp8", 1.0)):
-            key = name if temperature > 0 else name + "_greedy"
+        for name, temperature in (("llama3b", 1.0), ("llama8b", 1.0), ("llama8b", 0.7), ("qwen4b", 1.0), ("qwen4b", 0.0),
+                                  ("llama8b_30", 1.0), ("llama8b_2t", 1.0), ("batch32_2t", 1.0), ("batch32_fp8", 1.0)):
+            key = name if temperature == 1.0 else name + ("_greedy" if temperature == 0 else f"_t{temperature:g}")
             others[key] = time_other_workload(name, temperature, device, local, peaks)
     else:
         launches_main = args.steps * step.launches_per_step()

@@ -546,9 +546,6 @@ attention_pair_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
 {
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& sh = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    // The kernel after this one in the stream may be scheduled as soon as every CTA has got here; it
-    // waits for this grid's completion itself before it touches anything this grid reads or writes.
-
     const int warp = threadIdx.x >> 5;
     const uint32_t rank = cluster_ctarank();
 
