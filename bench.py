@@ -564,6 +564,7 @@ def run_ours(args, cfg):
         return
     peaks = measured_peaks()
     sm_count = step_mod.sm_count(step)
+    kname = step.attention_kernel_name()
     lens = attention_lens(cfg, plen, ms_attn * 1e-3 / cfg.L, clocks, peaks, sm_count)
     # the other workloads of the table (batch 1 shapes of the three model families, and one contemplate
     # row per node), each with its own clock record; one GPU only, after the main workload's memory is gone
@@ -582,7 +583,6 @@ def run_ours(args, cfg):
     else:
         launches_main = args.steps * step.launches_per_step()
     sbytes = step_bytes(cfg, plen, alen)
-    kname = step_mod.attention_kernel_name(cfg)
     cpu = oracle_sample(oracle_prepare(cfg)) if not args.no_cpu_baseline else None
     cpu_1t = oracle_one_thread(("tiny", "llama3b")) if not args.no_cpu_baseline else None
     tensor_bound = lens["bound"] == "tensor"

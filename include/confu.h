@@ -143,6 +143,13 @@ enum { CONFU_ATTENTION_AUTO = 0, CONFU_ATTENTION_GENERIC = 1, CONFU_ATTENTION_TE
 int confu_set_option(confu_ctx* ctx, int32_t option, int64_t value);
 
 /*
+ * The CONFU_ATTENTION_* path (never _AUTO) that confu_tree_plan and confu_tree_attention take for
+ * these dims under the context's current options, or a negative CONFU_ERR_* code where they would
+ * return it.  Host state only.
+ */
+int confu_attention_path(const confu_ctx* ctx, const confu_dims* dims);
+
+/*
  * Self-test of the bounded device-side wait (no counterpart in the paper): one warp waits, through
  * the same routine the attention kernels use, on a barrier that nothing arrives at; after limit_ns
  * (1 us .. 1 s) of wall clock the wait gives up and the kernel writes CONFU_ST_TIMEOUT to status[0]
@@ -200,7 +207,8 @@ int confu_tree_plan(confu_ctx* ctx, const confu_dims* dims,
  * and trees, or NULL to have the call build one in the workspace (then parent,
  * con_owner are read; otherwise they may be NULL).  Accumulation is fp32; bf16
  * inputs use the tensor-core path when D == 128 and Hq/Hkv <= 4; it takes the
- * query rows in groups of 64, so R > 64 streams the keys twice.
+ * query rows in groups of 64, so R > 64 streams the keys twice (the two groups walk
+ * the same keys at the same time: the second read is served by L2).
  * Needs the workspace.  All pointers device.  Ordinary stream order holds: the kernels are
  * launched as programmatic dependents (their blocks may be scheduled while the kernel before them
  * drains) but wait for all earlier work of the stream before their first global memory access,

@@ -27,7 +27,8 @@ EXPORTS = [
     "confu_last_cuda_error", "confu_plan_bytes", "confu_tree_plan", "confu_tree_attention",
     "confu_accept_workspace_bytes", "confu_tree_accept", "confu_kv_compact", "confu_kv_append",
     "confu_tree_accept_static_max_rows", "confu_tree_accept_static", "confu_set_paging",
-    "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_selftest_bounded_wait", "confu_set_kv_scales",
+    "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_attention_path",
+    "confu_selftest_bounded_wait", "confu_set_kv_scales",
 ]
 
 
@@ -55,7 +56,8 @@ def lib():
         L.confu_last_cuda_error.restype = C.c_char_p
         for n in ("confu_create", "confu_destroy", "confu_set_workspace", "confu_tree_plan", "confu_tree_attention",
                   "confu_tree_accept", "confu_kv_compact", "confu_kv_append", "confu_tree_accept_static", "confu_set_paging",
-                  "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_selftest_bounded_wait", "confu_set_kv_scales"):
+                  "confu_tree_accept_match", "confu_con_embedding", "confu_set_option", "confu_attention_path", "confu_selftest_bounded_wait",
+                  "confu_set_kv_scales"):
             getattr(L, n).restype = C.c_int
         _lib = L
     return _lib
@@ -128,6 +130,14 @@ def confu_set_kv_scales(ctx, k_scale, v_scale):
 
 def confu_set_option(ctx, option, value):
     _check("confu_set_option", lib().confu_set_option(ctx, C.c_int32(option), C.c_int64(value)))
+
+
+def confu_attention_path(ctx, dims):
+    """The ATTENTION_* path the library takes for these dims (never ATTENTION_AUTO); raises where the calls would fail."""
+    rc = int(lib().confu_attention_path(ctx, C.byref(dims)))
+    if rc < 0:
+        _check("confu_attention_path", rc)
+    return rc
 
 
 def confu_selftest_bounded_wait(ctx, limit_ns, status, stream=None):

@@ -8,7 +8,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libconfu.so")
 SOURCES = ["api.cu", "plan.cu", "attn_generic.cu", "attn_tc.cu", "attn_tc2.cu", "attn_fp8.cu", "combine.cu", "accept.cu", "accept_static.cu", "compact.cu", "moe.cu", "selftest.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "attn_tc.cuh"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(CSRC, "tc_walk.cuh"), os.path.join(ROOT, "include", "confu.h")]
+HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "attn_tc.cuh"), os.path.join(CSRC, "tc_ptx.cuh"), os.path.join(CSRC, "tc_walk.cuh"), os.path.join(CSRC, "combine.cuh"),
+           os.path.join(ROOT, "include", "confu.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

@@ -175,6 +175,14 @@ int confu_set_option(confu_ctx* ctx, int32_t option, int64_t value)
     }
 }
 
+int confu_attention_path(const confu_ctx* ctx, const confu_dims* dims)
+{
+    if (!ctx) return CONFU_ERR_ARG;
+    const int rc = check_dims(dims);
+    if (rc != CONFU_OK) return rc;
+    return resolve_attention_path(ctx, *dims);
+}
+
 int confu_selftest_bounded_wait(confu_ctx* ctx, int64_t limit_ns, int32_t* status, void* stream)
 {
     if (!ctx || !status) return CONFU_ERR_ARG;

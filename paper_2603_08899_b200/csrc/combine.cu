@@ -1,21 +1,10 @@
 // Merge of the split-KV partial results of the tensor-core attention kernel: a pair (sequence, kv
 // head, row group) whose key tiles were walked by several CTAs has one unnormalised partial (O, m,
 // l) per CTA; these kernels combine them into the output rows.
-#include "attn_tc.cuh"
+#include "combine.cuh"
 
 namespace confu {
 namespace tc {
-
-// Output row (b, r, head g * G + hl) and its lse as zeros, by one warp: what a sequence with a
-// malformed tree gets (the same as on the generic path).
-__device__ __forceinline__ void zero_row(const Params& prm, int b, int g, int r, int hl, int lane)
-{
-    const int R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
-    if (r >= R) return;
-    const int h = g * prm.G + hl;
-    reinterpret_cast<uint2*>(prm.out + (((size_t)b * R + r) * Hq + h) * kD)[lane] = make_uint2(0u, 0u);
-    if (prm.lse && lane == 0) prm.lse[((size_t)b * R + r) * Hq + h] = 0.f;
-}
 
 // Merge of the split-KV partials of one (sequence, kv head) pair, in CTA order (deterministic).
 // One block per (pair, M tile, 32 rows); a warp takes a row at a time (four rows in all), lane i the
@@ -86,73 +75,7 @@ __global__ void __launch_bounds__(32 * kCombineRowsPerBlock) combine_wide_kernel
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may start its prologue
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the attention kernel has completed
     const PlanView pv = plan_view(const_cast<void*>(prm.plan), prm.d.B);
-    const int pair = blockIdx.x, t = blockIdx.y;
-    // pairs: sequence major, then kv head, then row group
-    const int per_seq = prm.d.Hkv * prm.n_rg;
-    const int b = pair / per_seq, g = (pair % per_seq) / prm.n_rg, rg = pair % prm.n_rg;
-    const int nt = pv.tiles[b];
-    if (t >= prm.n_mt) return;
-    const int G = prm.G, R = prm.d.T + prm.d.C, Hq = prm.d.Hq;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int lane_row = blockIdx.z * kCombineRowsPerBlock + warp;
-    const int r = kGroupRows * rg + 32 * t + lane_row / G, hl = lane_row % G;
-    if (lane_row >= 32 * G || r >= R) return;
-    if (nt == 0) {                                      // malformed tree: no CTA worked on the pair; its rows read 0
-        zero_row(prm, b, g, r, hl, lane);
-        return;
-    }
-    const int64_t N = pv.hdr->n_tiles, n = pv.hdr->n_ctas / prm.n_rg;
-    // key tile q of (sequence, kv head) sits at position F + q of the cost line; position x belongs to lane
-    // floor(((x + 1) * n - 1) / N) of the n lanes, and row group rg of lane c is walked by CTA c * n_rg + rg
-    const int64_t F = pv.tile_base[b] + (int64_t)g * (nt + kPairOverheadTiles) + kPairOverheadTiles;
-    const int c_first = (int)(((F + 1) * n - 1) / N) * prm.n_rg + rg, c_last = (int)(((F + nt) * n - 1) / N) * prm.n_rg + rg;
-    if (c_first == c_last) return;                      // one CTA covered the pair and wrote the output itself
-    const int row = t * 128 + lane_row;
-    const int n_parts = (c_last - c_first) / prm.n_rg + 1;
-    const size_t slot_floats = partial_slot_bytes() / sizeof(float);
-    auto slot_of = [&](int p) {                         // part p of the pair: the partial slot of the p-th CTA that walked it
-        const int cta = c_first + p * prm.n_rg;
-        return prm.partials + (size_t)(2 * cta + (cta < c_last ? 1 : 0)) * slot_floats;
-    };
-    float M = -INFINITY;
-    for (int p = lane; p < n_parts; p += 32) M = fmaxf(M, slot_of(p)[(size_t)kPartRows * kPartD + row]);
-    M = warp_max(M);
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float L = 0.f;
-    for (int p0 = 0; p0 < n_parts; p0 += 32) {
-        float w = 0.f, wl = 0.f;                        // this lane's part of the group: weight, weight * sum
-        if (p0 + lane < n_parts) {
-            const float* ml = slot_of(p0 + lane) + (size_t)kPartRows * kPartD;
-            const float m = ml[row];
-            w = (m == -INFINITY) ? 0.f : ex2(m - M);
-            wl = w * ml[kPartRows + row];
-        }
-        L += warp_sum(wl);
-        const int n_grp = min(32, n_parts - p0);
-        for (int q0 = 0; q0 < n_grp; q0 += 8) {
-            float4 v[8];
-            float wq[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                wq[k] = __shfl_sync(0xffffffffu, w, (q0 + k) & 31);      // 0 past the last part
-                v[k] = q0 + k < n_grp ? reinterpret_cast<const float4*>(slot_of(p0 + q0 + k) + (size_t)row * kPartD)[lane]
-                                      : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                acc.x = fmaf(wq[k], v[k].x, acc.x); acc.y = fmaf(wq[k], v[k].y, acc.y);
-                acc.z = fmaf(wq[k], v[k].z, acc.z); acc.w = fmaf(wq[k], v[k].w, acc.w);
-            }
-        }
-    }
-    const float inv_l = 1.f / L;
-    const int h = g * G + hl;
-    __nv_bfloat16* orow = prm.out + (((size_t)b * R + r) * Hq + h) * kD;
-    uint2 pkt;
-    pkt.x = pack_bf16(acc.x * inv_l, acc.y * inv_l);
-    pkt.y = pack_bf16(acc.z * inv_l, acc.w * inv_l);
-    reinterpret_cast<uint2*>(orow)[lane] = pkt;
-    if (prm.lse && lane == 0) prm.lse[((size_t)b * R + r) * Hq + h] = (M + log2f(L)) * 0.6931471805599453f;
+    merge_row(prm, pv, blockIdx.x, blockIdx.y, blockIdx.z * kCombineRowsPerBlock + (threadIdx.x >> 5), threadIdx.x & 31);
 }
 
 cudaError_t launch_combine(const Params& prm, int sm_count, cudaStream_t st)

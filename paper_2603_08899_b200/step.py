@@ -117,7 +117,23 @@ class VerifyStep:
     def launches_per_step(self):
         """Kernels of this library launched by run(): plan + per layer attention + row statistics +
         walk + compaction."""
-        return 1 + attention_kernels_per_layer(self.cfg) * len(self.q) + 3
+        return 1 + self.attention_kernels_per_layer() * len(self.q) + 3
+
+    def attention_path(self):
+        """The library's choice of attention kernel for this step's dims (a binding.ATTENTION_* value)."""
+        return cb.confu_attention_path(self.ctx, self.dims)
+
+    def attention_kernel_name(self):
+        path = self.attention_path()
+        if path == cb.ATTENTION_GENERIC:
+            return "attention_generic_kernel"
+        if path == cb.ATTENTION_TENSOR_PAIR:
+            return "attention_pair_kernel"
+        return "attention_fp8_kernel" if self.cfg.kv_dtype == torch.float8_e4m3fn else "attention_tc_kernel"
+
+    def attention_kernels_per_layer(self):
+        """The tensor-core kernels are followed by the merge of the split pairs; the generic path is one kernel."""
+        return 2 if self.attention_path() in (cb.ATTENTION_TENSOR, cb.ATTENTION_TENSOR_PAIR) else 1
 
 
 def sm_count(step):
@@ -128,20 +144,3 @@ def sm_count(step):
 def uses_tensor_core_path(cfg):
     """Mirror of the library's dispatch rule: bf16 or E4M3 cache, head dim 128, at most 4 query heads per KV head."""
     return cfg.kv_dtype in (torch.bfloat16, torch.float8_e4m3fn) and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
-
-
-def attention_kernel_name(cfg):
-    """Mirror of the library's choice of attention kernel (CONFU_ATTENTION_AUTO)."""
-    if not uses_tensor_core_path(cfg):
-        return "attention_generic_kernel"
-    if cfg.kv_dtype == torch.float8_e4m3fn:
-        return "attention_fp8_kernel"
-    n_rg = (cfg.T + cfg.C + 63) // 64
-    sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count if torch.cuda.is_available() else 148
-    few_pairs = cfg.B * cfg.Hkv * n_rg <= sms // 2
-    return "attention_pair_kernel" if (cfg.T + cfg.C > 32 and few_pairs) else "attention_tc_kernel"
-
-
-def attention_kernels_per_layer(cfg):
-    """Tensor-core path: attention + split combine; generic path: one kernel."""
-    return 2 if uses_tensor_core_path(cfg) else 1
