@@ -139,8 +139,3 @@ class VerifyStep:
 def sm_count(step):
     """SM count of the step's device (one attention CTA per SM)."""
     return torch.cuda.get_device_properties(torch.device(step.dev)).multi_processor_count
-
-
-def uses_tensor_core_path(cfg):
-    """Mirror of the library's dispatch rule: bf16 or E4M3 cache, head dim 128, at most 4 query heads per KV head."""
-    return cfg.kv_dtype in (torch.bfloat16, torch.float8_e4m3fn) and cfg.D == 128 and cfg.Hq // cfg.Hkv <= 4 and cfg.S <= 128
