@@ -167,3 +167,45 @@ def test_quantising_append_is_bit_exact(gpu):
     untouched = torch.ones(n_slots, dtype=torch.bool)
     untouched[rows] = False
     assert (gk[untouched] == 0x11).all() and (gv[untouched] == 0x22).all()
+
+
+def test_fp8_full_size_workload_on_sampled_sequences():
+    """The full-size E4M3 workload of the benchmark, one layer, in the launch configuration the benchmark
+    times.  The oracle recomputes sampled rows of the longest, the shortest and one more sequence, each
+    from that sequence's own slice of the cache (widened exactly)."""
+    from paper_2603_08899_b200.step import VerifyStep
+    cfg = inputs.CONFIGS["batch32_fp8"]
+    parent, owner = inputs.trees(cfg)
+    plen = inputs.prefix_lens(cfg)
+    seq_start, n_slots = inputs.cache_layout(cfg, plen)
+    t = inputs.layer_tensors(cfg, 0, n_slots, device="cuda")
+    step = VerifyStep(cfg, n_slots)
+    out = torch.empty_like(t["q"])
+    lse = torch.empty(cfg.B, cfg.R, cfg.Hq, dtype=torch.float32, device="cuda")
+    tl = torch.zeros(1, device="cuda")
+    step.bind([t["q"]], [t["k_cache"]], [t["v_cache"]], [t["k_soft"]], [t["v_soft"]], [out], seq_start.cuda(),
+              plen.cuda(), parent.cuda(), owner.cuda(), tl, tl, tl, tl, kv_scales=[(t["k_scale"], t["v_scale"])])
+    step.run_attention([lse])
+    torch.cuda.synchronize()
+    assert (step.status == 0).all()
+    out_c, lse_c = out.cpu(), lse.cpu()
+    assert torch.isfinite(out_c.float()).all()
+    k_scale, v_scale = t["k_scale"].cpu(), t["v_scale"].cpu()
+    ks = ref.dequantize_cache(t["k_soft"].cpu(), k_scale)
+    vs = ref.dequantize_cache(t["v_soft"].cpu(), v_scale)
+    g = torch.Generator().manual_seed(11)
+    for b in sorted({int(plen.argmax()), int(plen.argmin()), 17}):
+        lo, n = int(seq_start[b]), int(plen[b]) + cfg.R
+        k = ref.dequantize_cache(t["k_cache"][lo:lo + n].cpu(), k_scale)
+        v = ref.dequantize_cache(t["v_cache"][lo:lo + n].cpu(), v_scale)
+        rows = torch.cat([torch.randint(0, cfg.R, (12,), generator=g), torch.tensor([0, cfg.T - 1, cfg.T, cfg.R - 1])])
+        heads = torch.randint(0, cfg.Hq, (rows.numel(),), generator=g)
+        sel = torch.stack([torch.zeros_like(rows), rows, heads], 1).to(torch.int32)
+        want, want_lse = ref.tree_attention_rows(t["q"][b:b + 1].cpu().to(torch.float64), k, v, torch.zeros(1, dtype=torch.int64),
+                                                 plen[b:b + 1], ks, vs, parent[b:b + 1], owner[b:b + 1], sel)
+        ref_max = want.abs().max().item()
+        for i, (_, r, h) in enumerate(sel.tolist()):
+            err = (out_c[b, r, h].double() - want[i]).abs().max().item()
+            assert err <= TOL_REL * ref_max, (b, r, h, err, ref_max)
+            assert abs(lse_c[b, r, h].item() - want_lse[i].item()) <= TOL_LSE, (b, r, h)
+    step.close()

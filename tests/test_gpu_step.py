@@ -83,7 +83,7 @@ def test_batched_ragged_step_reduced():
     assert exact + border == cfg.B and border <= 1
 
 
-@pytest.mark.parametrize("name", ["llama3b", "llama8b", "qwen4b", "batch32", "llama8b_2t"])
+@pytest.mark.parametrize("name", ["llama3b", "llama8b", "qwen4b", "batch32", "llama8b_2t", "llama8b_30", "batch32_2t"])
 def test_full_size_attention_on_sampled_rows(name):
     """The full-size workload of the benchmark, one layer, in the launch configuration the
     benchmark times; the oracle recomputes a sample of output rows one by one."""
