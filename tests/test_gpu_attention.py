@@ -57,6 +57,10 @@ CASES = {
     "bf16_one_pair_130_parts": _cfg(B=1, Hq=4, Hkv=1, prefix=16500, seed=57),
     # more pairs than SMs: whole pairs per CTA, few splits
     "bf16_many_short_sequences": _cfg(B=170, Hq=4, Hkv=2, prefix=(1, 260), seed=58),
+    # the same with two groups of 64 rows per pair (each share of the work is walked by two CTAs side by side),
+    # and one long pair of two row groups spread over all CTAs
+    "bf16_many_short_sequences_rows_80": _cfg(B=90, Hq=4, Hkv=2, T=40, C=40, prefix=(1, 260), max_depth=7, fanout=(1, 4), seed=59),
+    "bf16_one_pair_rows_100_many_parts": _cfg(B=1, Hq=4, Hkv=1, T=50, C=50, prefix=12000, max_depth=7, fanout=(1, 4), seed=60),
 }
 
 
