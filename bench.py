@@ -311,8 +311,8 @@ def spot_check(cfg, step, host):
 
 
 def time_other_workload(name, temperature, device, gpu_index, peaks, min_seconds=1.0):
-    """One more workload of the table, timed as replays of its captured graphs for at least min_seconds
-    (so that the clock sampler sees the load), its KV freed afterwards.  Returns the record that goes
+    """One more workload of the table, timed as replays of its captured step (one graph launch per step)
+    for at least min_seconds (so that the clock sampler sees the load), its KV freed afterwards.  Returns the record that goes
     under config.workloads[name]."""
     from paper_2603_08899_b200 import step as step_mod
     cfg, step, host = build_workload(inputs.CONFIGS[name], device, 0, temperature)
@@ -330,17 +330,25 @@ def time_other_workload(name, temperature, device, gpu_index, peaks, min_seconds
     e1.record()
     torch.cuda.synchronize()
     n = int(min(20000, max(20, min_seconds * 1e3 / max(e0.elapsed_time(e1) / 5, 1e-3))))
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n)]
+    # the parts of a step from replays as four graphs (a tenth as many), the step itself as one graph per step
+    n_parts = max(20, n // 10)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(n_parts)]
+    for i in range(n_parts):
+        step.replay(ev[i])
+    torch.cuda.synchronize()
+    ms_attn = statistics.mean(ev[i][1].elapsed_time(ev[i][2]) for i in range(n_parts))
+    ms_acc = statistics.mean(ev[i][2].elapsed_time(ev[i][3]) for i in range(n_parts))
+    ev_step = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
     sampler = ClockSampler(gpu_index)
     torch.cuda.synchronize()
     for i in range(n):
-        step.replay(ev[i])
+        ev_step[i].record()
+        step.replay_step()
+    ev_step[n].record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    ms = [ev[i][0].elapsed_time(ev[i][4]) for i in range(n)]
-    total_ms = ev[0][0].elapsed_time(ev[n - 1][4])
-    ms_attn = statistics.mean(ev[i][1].elapsed_time(ev[i][2]) for i in range(n))
-    ms_acc = statistics.mean(ev[i][2].elapsed_time(ev[i][3]) for i in range(n))
+    ms = [ev_step[i].elapsed_time(ev_step[i + 1]) for i in range(n)]
+    total_ms = ev_step[0].elapsed_time(ev_step[n])
     alen = step.accept_len.float().mean().item()
     sbytes = step_bytes(cfg, plen, alen) if temperature > 0 else \
         step_bytes(cfg, plen, alen) - cfg.B * cfg.T * cfg.V * step.tl.element_size()       # greedy reads the target matrix only
@@ -408,15 +416,16 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
     checked = spot_check(cfg, step, host) if rank == 0 else True
     status_ok = bool((step.status == 0).all().item())
-    # The timed steps replay the step's launches from CUDA graphs captured here (the same kernels with
-    # the same arguments; the host then issues 4 graph launches per step instead of 2 L + 4 kernels).
+    # The timed steps replay the step's launches from a CUDA graph captured here (the same kernels with
+    # the same arguments; the host then issues one graph launch per step instead of 2 L + 4 kernels).
     use_graph = not args.no_graph
     if use_graph:
         step.capture(1.0)
         for _ in range(2):
-            step.replay()
+            step.replay_step()
         torch.cuda.synchronize()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    ev_step = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     sampler = ClockSampler(local) if rank == 0 else None
     barrier()
     t_begin = torch.cuda.Event(enable_timing=True)
@@ -424,7 +433,8 @@ def run_ours(args, cfg):
     t_begin.record()
     for i in range(args.steps):
         if use_graph:
-            step.replay(ev[i])
+            ev_step[i].record()
+            step.replay_step()              # the whole step: one graph launch
             continue
         ev[i][0].record()
         step.run_plan()
@@ -435,14 +445,22 @@ def run_ours(args, cfg):
         ev[i][3].record()
         step.run_compact()
         ev[i][4].record()
+    ev_step[args.steps].record()
     t_end.record()
     barrier()
     clocks = sampler.stop() if sampler else None
+    if use_graph:
+        # the parts of a step (plan | attention | acceptance | compaction), timed apart from the headline:
+        # the same steps once more as four graphs with events between them
+        for i in range(args.steps):
+            step.replay(ev[i])
+        torch.cuda.synchronize()
     total_ms = max_over_ranks(t_begin.elapsed_time(t_end), dist, device)
     ms_step = total_ms / args.steps
     part = lambda a, b: statistics.mean(ev[i][a].elapsed_time(ev[i][b]) for i in range(args.steps))  # noqa: E731
     ms_plan, ms_attn, ms_acc, ms_cmp = part(0, 1), part(1, 2), part(2, 3), part(3, 4)
-    ms_each = [ev[i][0].elapsed_time(ev[i][4]) for i in range(args.steps)]
+    ms_each = [ev_step[i].elapsed_time(ev_step[i + 1]) for i in range(args.steps)] if use_graph else \
+        [ev[i][0].elapsed_time(ev[i][4]) for i in range(args.steps)]
     alen = step.accept_len.float().mean().item()
 
     def time_accept_variants():
@@ -572,7 +590,7 @@ def run_ours(args, cfg):
     if world == 1 and not args.no_other_workloads and args.config == "batch32":
         launches_main = args.steps * step.launches_per_step()
         step.close()
-        for name in ("q", "k", "v", "ks", "vs", "out", "tl", "dl", "graphs"):
+        for name in ("q", "k", "v", "ks", "vs", "out", "tl", "dl", "graphs", "graph_step"):
             setattr(step, name, None)
         torch.cuda.empty_cache()
         others = {}
@@ -598,7 +616,7 @@ def run_ours(args, cfg):
                    "l2": "inputs larger than L2 (every layer has its own KV; no flush needed)",
                    "parallelism": f"replicas x{world}, sequences sharded, no collective",
                    "parts_ms": {"plan": ms_plan, "attention": ms_attn, "accept": ms_acc, "compact": ms_cmp},
-                   "launch": "4 CUDA graphs per step (plan | L attention layers | acceptance | compaction)" if use_graph
+                   "launch": "1 CUDA graph per step; parts_ms from the same steps replayed as 4 graphs (plan | L attention layers | acceptance | compaction) after the timed region" if use_graph
                              else "kernel launches from the host, one by one",
                    "accept_rule": "ratio test, statistics of all rows (timed); variants timed apart: " \
                                   "lazy = same rule, rows on demand; match = sample-and-match, rows on demand",

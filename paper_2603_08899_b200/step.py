@@ -76,7 +76,8 @@ class VerifyStep:
 
     def capture(self, temperature=1.0, sibling_mode=1):
         """Record the step's launches once as four CUDA graphs (plan | attention layers | acceptance |
-        compaction) over the bound tensors; replay() then enqueues a step with four graph launches
+        compaction) over the bound tensors, and once more as a single graph; replay() then enqueues a
+        step with four graph launches (events can go between the parts), replay_step() with one,
         instead of 2 L + 4 kernel launches from the host.  Run the step once before capturing (the
         first call of each kernel sets function attributes, which a capture does not allow)."""
         parts = (self.run_plan, self.run_layers, lambda: self.run_accept(temperature, sibling_mode), self.run_compact)
@@ -86,6 +87,15 @@ class VerifyStep:
             with torch.cuda.graph(g):
                 fn()
             self.graphs.append(g)
+        # and the whole step as one graph: one launch from the host per step (replay_step)
+        self.graph_step = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph_step):
+            for fn in parts:
+                fn()
+
+    def replay_step(self):
+        """Enqueue one captured step on the current stream as a single graph launch."""
+        self.graph_step.replay()
 
     def replay(self, events=None):
         """Enqueue one captured step on the current stream; events: optional 5 CUDA events recorded
